@@ -1,0 +1,176 @@
+/*
+ * libdynbatch -- the parameter-server step of dynamic-batching BSP training
+ * (Tyagi & Sharma, "Taming Resource Heterogeneity In Distributed ML Training
+ * With Dynamic Batching"), as CUDA kernels for NVIDIA B200 (sm_100a) behind a
+ * plain C ABI.
+ *
+ * Conventions shared by every entry point
+ *   - "device" pointers are CUDA device memory owned by the caller; "host"
+ *     pointers are ordinary host memory.  The library allocates no device
+ *     memory: scratch space is a caller-provided workspace sized by the
+ *     matching *_workspace_bytes query.
+ *   - Device work is enqueued on `cuda_stream` (a cudaStream_t passed as
+ *     void*; NULL is the legacy default stream) and the call returns without
+ *     synchronising.  Host arrays (batch sizes, pointer tables) are consumed
+ *     before the call returns.
+ *   - Every call returns a db_status.  Arguments are validated before any
+ *     launch; on an error nothing has been enqueued and no output is touched.
+ *     Nothing throws, aborts or traps.  After DB_ERR_CUDA,
+ *     db_last_cuda_error() returns the runtime's message for this thread.
+ *   - NaN/Inf in the inputs propagate by IEEE rules; they are not checked.
+ */
+#ifndef DYNBATCH_H_
+#define DYNBATCH_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#pragma GCC visibility push(default)
+#endif
+
+typedef enum {
+    DB_OK = 0,
+    DB_ERR_NULL = 1,        /* a required pointer is NULL */
+    DB_ERR_ARG = 2,         /* a value is out of its documented range */
+    DB_ERR_UNSUPPORTED = 3, /* unknown dtype / configuration */
+    DB_ERR_INFEASIBLE = 4,  /* batch-size bounds cannot sum to the global batch */
+    DB_ERR_CUDA = 5         /* the CUDA runtime reported an error */
+} db_status;
+
+typedef enum {
+    DB_F32 = 0,  /* IEEE binary32 */
+    DB_BF16 = 1  /* bfloat16 (upper half of a binary32) */
+} db_dtype;
+
+/* Largest number of workers one call combines. */
+#define DB_MAX_K 64
+
+/* ------------------------------------------------------------------------
+ * Weighted aggregation + momentum-SGD update      (Section 3.1, Eq. 2-3;
+ * momentum optimizer of the ResNet-50 workload, Section 4)
+ *
+ * For every parameter j, in one pass over memory:
+ *     g    = sum_k lambda_k * grads[k][j],  lambda_k = b[k] / sum_i b[i]
+ *     v[j] = mu * v[j] + g
+ *     p[j] = p[j] - lr * v[j]
+ * and, optionally, grad_sqnorm = sum_j g^2.
+ *
+ * grads[k] is worker k's MEAN gradient over its b[k] samples.  The sum runs
+ * over k ascending with fp32 fused multiply-adds from a zero accumulator, so
+ * results are bit-reproducible and independent of launch geometry (the
+ * squared norm is reproducible for a fixed device and K).  Eq. 3's printed
+ * 1/K factor is not applied (with sum lambda = 1 it would break the stated
+ * equivalence with uniform batching); pass lr/K to get it.
+ *
+ *   grads          host array of K device pointers, each to N contiguous
+ *                  elements of grad_dtype; read-only.  A worker with
+ *                  b[k] == 0 has weight 0 and its buffer is never read.
+ *   b              host, K mini-batch sizes, each >= 0, sum > 0
+ *   K              1..DB_MAX_K
+ *   N              number of parameters, >= 0 (0: DB_OK, nothing enqueued)
+ *   params         device, N fp32, updated in place
+ *   momentum       device, N fp32, updated in place
+ *   lr, mu         finite learning rate and momentum coefficient
+ *   grad_sqnorm    device, one double, or NULL to skip the norm
+ *   workspace      device scratch of >= db_aggregate_workspace_bytes(K, N)
+ *                  bytes, 16-byte aligned; needs no initialisation; may be
+ *                  NULL when grad_sqnorm is NULL.  Calls that may overlap on
+ *                  the device need distinct workspaces.
+ *
+ * Any pointer alignment (down to the element size) and any N are accepted;
+ * the 128-bit path is taken when params, momentum and all gradient buffers
+ * reach a 16-byte boundary after the same number of leading elements,
+ * otherwise an element-wise kernel runs.  Gradient buffers must not overlap
+ * params or momentum, nor params momentum (DB_ERR_ARG).
+ *
+ * db_aggregate_update is the fp32, no-norm, default-stream short form.
+ * ------------------------------------------------------------------------ */
+db_status db_aggregate_update(const float* const* grads, const int32_t* b,
+                              int32_t K, int64_t N, float* params,
+                              float* momentum, float lr, float mu);
+
+db_status db_aggregate_update_ex(const void* const* grads, db_dtype grad_dtype,
+                                 const int32_t* b, int32_t K, int64_t N,
+                                 float* params, float* momentum, float lr,
+                                 float mu, double* grad_sqnorm, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream);
+
+size_t db_aggregate_workspace_bytes(int32_t K, int64_t N);
+
+/* ------------------------------------------------------------------------
+ * Ragged per-worker gradient of a linear-softmax classifier
+ *
+ * The model on which the batch-proportional weighting of Eq. 2 is checked
+ * against the gradient of the whole global batch (Section 3.1: the weights
+ * keep variable batching equivalent to uniform batching).  For worker i with
+ * b_i samples:
+ *     Z = X W;  P = softmax over each row of Z;  G = X^T (P - Y) / b_i
+ * with Y the one-hot labels; no bias; loss = mean cross-entropy.
+ *
+ *   X     device [b_i, D] row-major fp32
+ *   y     device [b_i] int32 labels in [0, C) (a label outside the range
+ *         contributes no one-hot term and a zero loss; not an error)
+ *   W     device [D, C] row-major fp32
+ *   b_i   1..65535,  D >= 1,  C >= 1
+ *   G     device [D, C] row-major fp32, overwritten
+ *   loss  device, one float (mean cross-entropy), or NULL
+ *   workspace  device scratch of >= db_worker_grad_workspace_bytes(b_i, D, C)
+ *         bytes, 16-byte aligned, uninitialised
+ * X, W, G must be 16-byte aligned when D and C are multiples of 4 (they are
+ * for any whole allocation); other shapes take element-wise loads.
+ * ------------------------------------------------------------------------ */
+db_status db_worker_grad(const float* X, const int32_t* y, const float* W,
+                         int32_t b_i, int32_t D, int32_t C, float* G,
+                         float* loss, void* workspace, size_t workspace_bytes,
+                         void* cuda_stream);
+
+size_t db_worker_grad_workspace_bytes(int32_t b_i, int32_t D, int32_t C);
+
+/* ------------------------------------------------------------------------
+ * Proportional batch-size controller, host side   (Section 3.3, Eq. 4-5)
+ *
+ * One adjustment from per-worker throughputs X_k (samples per unit time):
+ *     t_k = b_k / X_k;  tbar = mean_k t_k;  Db_k = -X_k (t_k - tbar)   (Eq. 4)
+ *     bt_k = b_k + kp * Db_k                                           (Eq. 5)
+ * kp = 1 is the paper's rule (equivalently b_k * tbar / t_k); kp in (0,1)
+ * damps it.  The targets are rescaled so that the global batch sum_k b_k is
+ * unchanged (the invariant Section 3.2 states for variable batching), then
+ * made integer within [b_min_k, b_max_k] (bounds: Section 3.3.1) by the
+ * largest-remainder rule: start from floor, hand missing units to the worker
+ * furthest below its target (ties: lowest index), take surplus units from
+ * the worker furthest above.  All arithmetic is IEEE fp64 in a fixed order,
+ * so the integer result is deterministic.
+ *
+ *   b            host, K batch sizes >= 0 with sum > 0; overwritten on DB_OK
+ *   throughputs  host, K finite values > 0
+ *   K            1..DB_MAX_K
+ *   kp           0 < kp <= 1
+ *   b_min,b_max  host, K each, or NULL for 1 and sum(b); 0 <= min <= max
+ * DB_ERR_INFEASIBLE (b untouched) if the bounds cannot sum to sum(b).
+ * ------------------------------------------------------------------------ */
+db_status db_controller_step(int32_t* b, const double* throughputs, int32_t K,
+                             double kp);
+
+db_status db_controller_step_ex(int32_t* b, const double* throughputs,
+                                int32_t K, double kp, const int32_t* b_min,
+                                const int32_t* b_max);
+
+/* Static text for a status code. */
+const char* db_status_string(db_status s);
+
+/* Message of the last CUDA error seen by this thread ("" if none). */
+const char* db_last_cuda_error(void);
+
+#if defined(__GNUC__)
+#pragma GCC visibility pop
+#endif
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DYNBATCH_H_ */

@@ -1,0 +1,163 @@
+"""Thin ctypes binding of libdynbatch (argument marshalling only).
+
+Every function has the name and meaning of the C entry point declared in
+include/dynbatch.h; tensors are torch tensors used purely as device memory
+(`data_ptr()`), and the stream is torch's current stream unless given.  All
+arithmetic runs inside the CUDA library: there is no Python or CPU fallback,
+and a missing shared library is an error, not a reason to compute elsewhere.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_char_p, c_double, c_float, c_int32, c_int64, c_size_t, c_void_p
+from typing import Optional, Sequence
+
+import torch
+
+DB_OK, DB_ERR_NULL, DB_ERR_ARG, DB_ERR_UNSUPPORTED, DB_ERR_INFEASIBLE, DB_ERR_CUDA = range(6)
+DB_F32, DB_BF16 = 0, 1
+DB_MAX_K = 64
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libdynbatch.so")
+
+_lib = None
+
+
+class DynbatchError(RuntimeError):
+    """A libdynbatch call returned a status other than DB_OK."""
+
+    def __init__(self, status: int, message: str):
+        super().__init__(f"libdynbatch status {status}: {message}")
+        self.status = status
+
+
+_SIGNATURES = {
+    "db_aggregate_update": (c_int32, [c_void_p, c_void_p, c_int32, c_int64, c_void_p, c_void_p,
+                                      c_float, c_float]),
+    "db_aggregate_update_ex": (c_int32, [c_void_p, c_int32, c_void_p, c_int32, c_int64, c_void_p,
+                                         c_void_p, c_float, c_float, c_void_p, c_void_p, c_size_t,
+                                         c_void_p]),
+    "db_aggregate_workspace_bytes": (c_size_t, [c_int32, c_int64]),
+    "db_worker_grad": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p,
+                                 c_void_p, c_void_p, c_size_t, c_void_p]),
+    "db_worker_grad_workspace_bytes": (c_size_t, [c_int32, c_int32, c_int32]),
+    "db_controller_step": (c_int32, [c_void_p, c_void_p, c_int32, c_double]),
+    "db_controller_step_ex": (c_int32, [c_void_p, c_void_p, c_int32, c_double, c_void_p, c_void_p]),
+    "db_status_string": (c_char_p, [c_int32]),
+    "db_last_cuda_error": (c_char_p, []),
+}
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2305_12213_b200.build`. "
+                "libdynbatch has no CPU fallback.")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def _check(status: int) -> None:
+    if status != DB_OK:
+        L = lib()
+        msg = L.db_status_string(status).decode()
+        if status == DB_ERR_CUDA:
+            msg += ": " + L.db_last_cuda_error().decode()
+        raise DynbatchError(status, msg)
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def _i32_array(values: Sequence[int]):
+    return (c_int32 * len(values))(*[int(x) for x in values])
+
+
+def _dev_ptr(t: Optional[torch.Tensor], dtype: torch.dtype, name: str) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"{name} must be a contiguous CUDA tensor of {dtype}")
+    return t.data_ptr()
+
+
+def aggregate_workspace_bytes(K: int, N: int) -> int:
+    return int(lib().db_aggregate_workspace_bytes(int(K), int(N)))
+
+
+def aggregate_update(grads: Sequence[torch.Tensor], b: Sequence[int], params: torch.Tensor,
+                     momentum: torch.Tensor, lr: float, mu: float,
+                     grad_sqnorm: Optional[torch.Tensor] = None,
+                     workspace: Optional[torch.Tensor] = None,
+                     stream: Optional[torch.cuda.Stream] = None, N: Optional[int] = None) -> None:
+    """db_aggregate_update_ex: fused weighted aggregation + momentum-SGD update, in place.
+
+    grads: K CUDA tensors (all float32 or all bfloat16) of N elements; b: K batch sizes;
+    params, momentum: float32 CUDA tensors; grad_sqnorm: optional float64 CUDA tensor of one
+    element; workspace: uint8 CUDA tensor of aggregate_workspace_bytes(K, N) when the norm is wanted.
+    """
+    K = len(grads)
+    if len(b) != K:
+        raise ValueError("len(b) != len(grads)")
+    gdt = grads[0].dtype
+    if gdt == torch.float32:
+        code = DB_F32
+    elif gdt == torch.bfloat16:
+        code = DB_BF16
+    else:
+        raise TypeError("gradients must be float32 or bfloat16")
+    n = int(params.numel() if N is None else N)
+    table = (c_void_p * K)(*[_dev_ptr(g, gdt, "grads[k]") for g in grads])
+    _check(lib().db_aggregate_update_ex(
+        ctypes.cast(table, c_void_p), code, ctypes.cast(_i32_array(b), c_void_p), K, n,
+        _dev_ptr(params, torch.float32, "params"), _dev_ptr(momentum, torch.float32, "momentum"),
+        float(lr), float(mu), _dev_ptr(grad_sqnorm, torch.float64, "grad_sqnorm"),
+        None if workspace is None else workspace.data_ptr(),
+        0 if workspace is None else workspace.numel() * workspace.element_size(),
+        _stream_ptr(stream)))
+
+
+def worker_grad_workspace_bytes(b_i: int, D: int, C: int) -> int:
+    return int(lib().db_worker_grad_workspace_bytes(int(b_i), int(D), int(C)))
+
+
+def worker_grad(X: torch.Tensor, y: torch.Tensor, W: torch.Tensor, G: torch.Tensor,
+                loss: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                stream: Optional[torch.cuda.Stream] = None) -> None:
+    """db_worker_grad: G = X^T (softmax(X W) - onehot(y)) / b_i, optional mean cross-entropy."""
+    b_i, D = X.shape
+    D2, C = W.shape
+    if D2 != D or tuple(G.shape) != (D, C) or y.numel() != b_i:
+        raise ValueError("shape mismatch")
+    _check(lib().db_worker_grad(
+        _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.int32, "y"), _dev_ptr(W, torch.float32, "W"),
+        b_i, D, C, _dev_ptr(G, torch.float32, "G"), _dev_ptr(loss, torch.float32, "loss"),
+        None if workspace is None else workspace.data_ptr(),
+        0 if workspace is None else workspace.numel() * workspace.element_size(),
+        _stream_ptr(stream)))
+
+
+def controller_step(b: Sequence[int], throughputs: Sequence[float], kp: float,
+                    b_min: Optional[Sequence[int]] = None,
+                    b_max: Optional[Sequence[int]] = None) -> list:
+    """db_controller_step_ex: one proportional-control adjustment; returns the new batch sizes."""
+    K = len(b)
+    if len(throughputs) != K:
+        raise ValueError("len(throughputs) != len(b)")
+    arr = _i32_array(b)
+    xs = (c_double * K)(*[float(x) for x in throughputs])
+    lo = None if b_min is None else ctypes.cast(_i32_array(b_min), c_void_p)
+    hi = None if b_max is None else ctypes.cast(_i32_array(b_max), c_void_p)
+    _check(lib().db_controller_step_ex(ctypes.cast(arr, c_void_p), ctypes.cast(xs, c_void_p), K,
+                                       float(kp), lo, hi))
+    return list(arr)

@@ -1,0 +1,402 @@
+// Fused K-way weighted gradient aggregation + momentum-SGD update
+// (Section 3.1, Eq. 2-3; momentum optimizer of Section 4's ResNet-50 workload).
+//
+// One pass over HBM: each thread owns one 16-byte vector position per step,
+// issues the loads of all K gradient slices and of the parameter/momentum
+// vectors before the first use, folds the slices with fp32 FMAs in worker
+// order, applies v = mu v + g, p = p - lr v and streams both back.  Nothing
+// else touches N-sized data; the squared gradient norm rides along in
+// registers.  The grid is persistent (a multiple of the SM count) and walks
+// the arrays tile by tile so that all SMs sweep the same DRAM pages together.
+#include <cuda_bf16.h>
+
+#include <cstdint>
+
+#include "common.h"
+
+namespace dynbatch {
+namespace {
+
+constexpr int kBlock = 256;
+constexpr int kMaxFixedK = 16;   // K up to here gets a fully unrolled kernel
+constexpr int kChunk = 8;        // gradient slices loaded per round beyond that
+
+struct AggArgs {
+    const void* g[DB_MAX_K];  // active workers' gradient buffers
+    float lambda[DB_MAX_K];   // their weights b_k / sum b
+    float* p;
+    float* v;
+    double* partials;         // one per CTA (norm only)
+    unsigned int* ticket;     // CTA arrival counter, zero at launch (norm only)
+    double* sq_out;
+    long long n;              // elements
+    long long head;           // leading elements before the first 16-byte boundary
+    long long nvec;           // whole vectors after the head
+    float lr, mu;
+    int K;
+};
+
+// Raw 16-byte gradient vector and its widening to fp32 lanes.
+template <typename GT> struct GradVec;
+
+template <> struct GradVec<float> {
+    static constexpr int kLanes = 4;
+    using Raw = float4;
+    static __device__ __forceinline__ Raw load(const void* base, long long head, long long vi) {
+        return __ldcs(reinterpret_cast<const float4*>(static_cast<const float*>(base) + head) + vi);
+    }
+    static __device__ __forceinline__ void widen(const Raw& r, float (&x)[4]) {
+        x[0] = r.x; x[1] = r.y; x[2] = r.z; x[3] = r.w;
+    }
+    static __device__ __forceinline__ float scalar(const void* base, long long j) {
+        return __ldcs(static_cast<const float*>(base) + j);
+    }
+};
+
+template <> struct GradVec<__nv_bfloat16> {
+    static constexpr int kLanes = 8;
+    using Raw = uint4;
+    static __device__ __forceinline__ Raw load(const void* base, long long head, long long vi) {
+        return __ldcs(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(base) + head) + vi);
+    }
+    // bf16 is the high half of a binary32: widening is a shift, exact.
+    static __device__ __forceinline__ void widen(const Raw& r, float (&x)[8]) {
+        x[0] = __uint_as_float(r.x << 16); x[1] = __uint_as_float(r.x & 0xffff0000u);
+        x[2] = __uint_as_float(r.y << 16); x[3] = __uint_as_float(r.y & 0xffff0000u);
+        x[4] = __uint_as_float(r.z << 16); x[5] = __uint_as_float(r.z & 0xffff0000u);
+        x[6] = __uint_as_float(r.w << 16); x[7] = __uint_as_float(r.w & 0xffff0000u);
+    }
+    static __device__ __forceinline__ float scalar(const void* base, long long j) {
+        const uint16_t h = __ldcs(static_cast<const uint16_t*>(base) + j);
+        return __uint_as_float(static_cast<uint32_t>(h) << 16);
+    }
+};
+
+// Block-wide sum of doubles in a fixed order (xor tree in the warp, warps in order).
+__device__ __forceinline__ double block_sum(double x, double* smem) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();
+    if (lane == 0) smem[warp] = x;
+    __syncthreads();
+    double s = 0.0;
+    if (threadIdx.x == 0) {
+        for (int w = 0; w < kBlock / 32; ++w) s += smem[w];
+    }
+    return s;  // valid in thread 0
+}
+
+// Publishes this CTA's partial; the last CTA to arrive folds all partials in
+// index order.  No CTA ever waits on another: arrival order is taken from an
+// atomic ticket, so the kernel cannot spin.
+__device__ __forceinline__ void finish_norm(const AggArgs& a, double sq) {
+    __shared__ double smem[kBlock / 32];
+    __shared__ bool is_last;
+    const double s = block_sum(sq, smem);
+    if (threadIdx.x == 0) {
+        a.partials[blockIdx.x] = s;
+        __threadfence();
+        const unsigned int t = atomicAdd(a.ticket, 1u);
+        is_last = (t == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    double acc = 0.0;
+    for (unsigned int i = threadIdx.x; i < gridDim.x; i += kBlock)
+        acc += __ldcg(a.partials + i);
+    const double total = block_sum(acc, smem);
+    if (threadIdx.x == 0) *a.sq_out = total;
+}
+
+// One element, any alignment: the same FMA chain as the vector body.
+template <typename GT, bool NORM>
+__device__ __forceinline__ void update_scalar(const AggArgs& a, int K, long long j, double& sq) {
+    float g = 0.0f;
+    for (int k = 0; k < K; ++k) g = fmaf(a.lambda[k], GradVec<GT>::scalar(a.g[k], j), g);
+    const float vn = fmaf(a.mu, a.v[j], g);
+    a.v[j] = vn;
+    a.p[j] = fmaf(-a.lr, vn, a.p[j]);
+    if (NORM) sq += static_cast<double>(g * g);
+}
+
+// Momentum update of the `kLanes` elements at vector index vi.
+template <int kLanes, bool NORM>
+__device__ __forceinline__ void apply_update(const AggArgs& a, long long vi, const float (&g)[kLanes],
+                                             const float4 (&pv)[kLanes / 4], const float4 (&vv)[kLanes / 4],
+                                             double& sq) {
+    float4* pp = reinterpret_cast<float4*>(a.p + a.head) + vi * (kLanes / 4);
+    float4* vp = reinterpret_cast<float4*>(a.v + a.head) + vi * (kLanes / 4);
+    float part = 0.0f;
+#pragma unroll
+    for (int q = 0; q < kLanes / 4; ++q) {
+        float4 vn, pn;
+        vn.x = fmaf(a.mu, vv[q].x, g[4 * q + 0]);
+        vn.y = fmaf(a.mu, vv[q].y, g[4 * q + 1]);
+        vn.z = fmaf(a.mu, vv[q].z, g[4 * q + 2]);
+        vn.w = fmaf(a.mu, vv[q].w, g[4 * q + 3]);
+        pn.x = fmaf(-a.lr, vn.x, pv[q].x);
+        pn.y = fmaf(-a.lr, vn.y, pv[q].y);
+        pn.z = fmaf(-a.lr, vn.z, pv[q].z);
+        pn.w = fmaf(-a.lr, vn.w, pv[q].w);
+        __stcs(vp + q, vn);
+        __stcs(pp + q, pn);
+        if (NORM) {
+#pragma unroll
+            for (int l = 0; l < 4; ++l) part = fmaf(g[4 * q + l], g[4 * q + l], part);
+        }
+    }
+    if (NORM) sq += static_cast<double>(part);
+}
+
+// KT > 0: exactly KT workers, fully unrolled.  KT == 0: a.K workers, kChunk at a time.
+template <typename GT, int KT, int UNROLL, bool NORM>
+__global__ void __launch_bounds__(kBlock)
+agg_vec_kernel(const __grid_constant__ AggArgs a) {
+    using GV = GradVec<GT>;
+    using Raw = typename GV::Raw;
+    constexpr int kLanes = GV::kLanes;
+    constexpr int kQuads = kLanes / 4;
+    const int K = KT > 0 ? KT : a.K;
+    double sq = 0.0;
+
+    const long long tile = static_cast<long long>(kBlock) * UNROLL;
+    const long long step = static_cast<long long>(gridDim.x) * tile;
+    for (long long base = static_cast<long long>(blockIdx.x) * tile; base < a.nvec; base += step) {
+        long long vi[UNROLL];
+        bool ok[UNROLL];
+        float4 pv[UNROLL][kQuads], vv[UNROLL][kQuads];
+        float g[UNROLL][kLanes];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            vi[u] = base + u * kBlock + threadIdx.x;
+            ok[u] = vi[u] < a.nvec;
+#pragma unroll
+            for (int l = 0; l < kLanes; ++l) g[u][l] = 0.0f;
+        }
+        if (KT > 0) {
+            Raw raw[UNROLL][KT > 0 ? KT : 1];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                if (!ok[u]) continue;
+#pragma unroll
+                for (int k = 0; k < KT; ++k) raw[u][k] = GV::load(a.g[k], a.head, vi[u]);
+#pragma unroll
+                for (int q = 0; q < kQuads; ++q) {
+                    pv[u][q] = __ldcs(reinterpret_cast<const float4*>(a.p + a.head) + vi[u] * kQuads + q);
+                    vv[u][q] = __ldcs(reinterpret_cast<const float4*>(a.v + a.head) + vi[u] * kQuads + q);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                if (!ok[u]) continue;
+#pragma unroll
+                for (int k = 0; k < KT; ++k) {
+                    float x[kLanes];
+                    GV::widen(raw[u][k], x);
+#pragma unroll
+                    for (int l = 0; l < kLanes; ++l) g[u][l] = fmaf(a.lambda[k], x[l], g[u][l]);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                if (!ok[u]) continue;
+#pragma unroll
+                for (int q = 0; q < kQuads; ++q) {
+                    pv[u][q] = __ldcs(reinterpret_cast<const float4*>(a.p + a.head) + vi[u] * kQuads + q);
+                    vv[u][q] = __ldcs(reinterpret_cast<const float4*>(a.v + a.head) + vi[u] * kQuads + q);
+                }
+                for (int k0 = 0; k0 < K; k0 += kChunk) {
+                    Raw raw[kChunk];
+#pragma unroll
+                    for (int i = 0; i < kChunk; ++i)
+                        if (k0 + i < K) raw[i] = GV::load(a.g[k0 + i], a.head, vi[u]);
+#pragma unroll
+                    for (int i = 0; i < kChunk; ++i) {
+                        if (k0 + i < K) {
+                            float x[kLanes];
+                            GV::widen(raw[i], x);
+#pragma unroll
+                            for (int l = 0; l < kLanes; ++l)
+                                g[u][l] = fmaf(a.lambda[k0 + i], x[l], g[u][l]);
+                        }
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u)
+            if (ok[u]) apply_update<kLanes, NORM>(a, vi[u], g[u], pv[u], vv[u], sq);
+    }
+
+    // ragged ends: fewer than kLanes elements on either side of the vector body
+    if (blockIdx.x == 0) {
+        const long long tail0 = a.head + a.nvec * kLanes;
+        if (threadIdx.x < a.head) update_scalar<GT, NORM>(a, K, threadIdx.x, sq);
+        if (tail0 + threadIdx.x < a.n) update_scalar<GT, NORM>(a, K, tail0 + threadIdx.x, sq);
+    }
+    if (NORM) finish_norm(a, sq);
+}
+
+// Element-wise kernel for buffers whose 16-byte boundaries do not line up.
+template <typename GT, bool NORM>
+__global__ void __launch_bounds__(kBlock)
+agg_scalar_kernel(const __grid_constant__ AggArgs a) {
+    double sq = 0.0;
+    const long long step = static_cast<long long>(gridDim.x) * kBlock;
+    for (long long j = static_cast<long long>(blockIdx.x) * kBlock + threadIdx.x; j < a.n; j += step)
+        update_scalar<GT, NORM>(a, a.K, j, sq);
+    if (NORM) finish_norm(a, sq);
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+constexpr size_t kTicketBytes = 256;  // ticket word, padded so the partials stay aligned
+
+using KernelFn = void (*)(const AggArgs);
+
+template <typename GT, int KT, bool NORM>
+KernelFn pick_unroll(int* unroll_out) {
+    // enough 16-byte loads in flight per thread: about 12-16 across the K+2 streams
+    constexpr int kStreams = (KT > 0 ? KT : kChunk) + 2 * GradVec<GT>::kLanes / 4;
+    constexpr int kUnroll = kStreams <= 4 ? 4 : (kStreams <= 8 ? 2 : 1);
+    *unroll_out = kUnroll;
+    return agg_vec_kernel<GT, KT, kUnroll, NORM>;
+}
+
+template <typename GT, bool NORM>
+KernelFn pick_vec_kernel(int K, int* unroll_out) {
+    switch (K) {
+#define DB_CASE(n) case n: return pick_unroll<GT, n, NORM>(unroll_out);
+        DB_CASE(1) DB_CASE(2) DB_CASE(3) DB_CASE(4) DB_CASE(5) DB_CASE(6) DB_CASE(7) DB_CASE(8)
+        DB_CASE(9) DB_CASE(10) DB_CASE(11) DB_CASE(12) DB_CASE(13) DB_CASE(14) DB_CASE(15) DB_CASE(16)
+#undef DB_CASE
+        default: return pick_unroll<GT, 0, NORM>(unroll_out);
+    }
+}
+
+bool ranges_overlap(const void* a, size_t abytes, const void* b, size_t bbytes) {
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return a0 < b0 + bbytes && b0 < a0 + abytes;
+}
+
+int grid_for(KernelFn fn, long long work_items_per_cta, long long work_items) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kBlock, 0) != cudaSuccess || per_sm < 1)
+        per_sm = 1;
+    const long long resident = static_cast<long long>(sm_count()) * per_sm;
+    long long need = (work_items + work_items_per_cta - 1) / work_items_per_cta;
+    if (need < 1) need = 1;
+    return static_cast<int>(need < resident ? need : resident);
+}
+
+}  // namespace
+}  // namespace dynbatch
+
+extern "C" size_t db_aggregate_workspace_bytes(int32_t K, int64_t N) {
+    (void)K; (void)N;
+    // ticket + one double per CTA; CTAs never exceed SMs x resident blocks (<= 32 per SM)
+    return dynbatch::kTicketBytes + sizeof(double) * 32 * static_cast<size_t>(dynbatch::sm_count());
+}
+
+extern "C" db_status db_aggregate_update_ex(const void* const* grads, db_dtype grad_dtype,
+                                            const int32_t* b, int32_t K, int64_t N,
+                                            float* params, float* momentum, float lr, float mu,
+                                            double* grad_sqnorm, void* workspace,
+                                            size_t workspace_bytes, void* cuda_stream) {
+    using namespace dynbatch;
+    if (!grads || !b) return DB_ERR_NULL;
+    if (K < 1 || K > DB_MAX_K || N < 0) return DB_ERR_ARG;
+    if (grad_dtype != DB_F32 && grad_dtype != DB_BF16) return DB_ERR_UNSUPPORTED;
+    if (!isfinite(lr) || !isfinite(mu)) return DB_ERR_ARG;
+    long long total = 0;
+    for (int k = 0; k < K; ++k) {
+        if (b[k] < 0) return DB_ERR_ARG;
+        total += b[k];
+    }
+    if (total <= 0) return DB_ERR_ARG;
+    if (N == 0) return DB_OK;
+    if (!params || !momentum) return DB_ERR_NULL;
+    const size_t gsize = grad_dtype == DB_F32 ? 4 : 2;
+    const size_t state_bytes = static_cast<size_t>(N) * 4, grad_bytes = static_cast<size_t>(N) * gsize;
+    if (reinterpret_cast<uintptr_t>(params) % 4 || reinterpret_cast<uintptr_t>(momentum) % 4) return DB_ERR_ARG;
+    if (ranges_overlap(params, state_bytes, momentum, state_bytes)) return DB_ERR_ARG;
+
+    AggArgs a{};
+    int active = 0;
+    for (int k = 0; k < K; ++k) {
+        if (b[k] == 0) continue;  // weight 0: the buffer is not read
+        if (!grads[k]) return DB_ERR_NULL;
+        if (reinterpret_cast<uintptr_t>(grads[k]) % gsize) return DB_ERR_ARG;
+        if (ranges_overlap(grads[k], grad_bytes, params, state_bytes) ||
+            ranges_overlap(grads[k], grad_bytes, momentum, state_bytes))
+            return DB_ERR_ARG;
+        a.g[active] = grads[k];
+        a.lambda[active] = static_cast<float>(static_cast<double>(b[k]) / static_cast<double>(total));
+        ++active;
+    }
+    a.K = active;
+    a.p = params;
+    a.v = momentum;
+    a.n = N;
+    a.lr = lr;
+    a.mu = mu;
+
+    const bool norm = grad_sqnorm != nullptr;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (norm) {
+        if (!workspace) return DB_ERR_NULL;
+        if (reinterpret_cast<uintptr_t>(workspace) % 16 || workspace_bytes < db_aggregate_workspace_bytes(K, N))
+            return DB_ERR_ARG;
+        a.ticket = static_cast<unsigned int*>(workspace);
+        a.partials = reinterpret_cast<double*>(static_cast<char*>(workspace) + kTicketBytes);
+        a.sq_out = grad_sqnorm;
+    }
+
+    // Leading elements until params reaches a 16-byte boundary; the vector body
+    // needs momentum and every gradient buffer on a boundary at the same element.
+    const int lanes = grad_dtype == DB_F32 ? 4 : 8;
+    long long head = static_cast<long long>(((16 - reinterpret_cast<uintptr_t>(params) % 16) % 16) / 4);
+    bool vector_ok = (reinterpret_cast<uintptr_t>(momentum) + head * 4) % 16 == 0;
+    if (vector_ok && grad_dtype == DB_BF16) {
+        // bf16 vectors hold 8 elements: pick the head in {head, head + 4} that aligns the gradients
+        const uintptr_t g0 = reinterpret_cast<uintptr_t>(a.g[0]);
+        if ((g0 + head * 2) % 16 != 0) head += 4;
+    }
+    for (int k = 0; vector_ok && k < active; ++k)
+        vector_ok = (reinterpret_cast<uintptr_t>(a.g[k]) + head * gsize) % 16 == 0;
+    if (head > N) head = N;
+    a.head = head;
+    a.nvec = (N - head) / lanes;
+
+    KernelFn fn;
+    int grid;
+    if (vector_ok) {
+        int unroll = 1;
+        if (grad_dtype == DB_F32)
+            fn = norm ? pick_vec_kernel<float, true>(active, &unroll) : pick_vec_kernel<float, false>(active, &unroll);
+        else
+            fn = norm ? pick_vec_kernel<__nv_bfloat16, true>(active, &unroll)
+                      : pick_vec_kernel<__nv_bfloat16, false>(active, &unroll);
+        grid = grid_for(fn, static_cast<long long>(kBlock) * unroll, a.nvec);
+    } else {
+        if (grad_dtype == DB_F32)
+            fn = norm ? agg_scalar_kernel<float, true> : agg_scalar_kernel<float, false>;
+        else
+            fn = norm ? agg_scalar_kernel<__nv_bfloat16, true> : agg_scalar_kernel<__nv_bfloat16, false>;
+        grid = grid_for(fn, kBlock, N);
+    }
+    if (norm) DB_CUDA_TRY(cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), stream));
+    fn<<<grid, kBlock, 0, stream>>>(a);
+    DB_CUDA_TRY(cudaGetLastError());
+    return DB_OK;
+}
+
+extern "C" db_status db_aggregate_update(const float* const* grads, const int32_t* b, int32_t K,
+                                         int64_t N, float* params, float* momentum, float lr, float mu) {
+    return db_aggregate_update_ex(reinterpret_cast<const void* const*>(grads), DB_F32, b, K, N, params,
+                                  momentum, lr, mu, nullptr, nullptr, 0, nullptr);
+}

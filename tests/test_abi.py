@@ -1,0 +1,178 @@
+"""CPU-only checks of the C-ABI library: it loads, exports what the header declares,
+validates arguments before touching the GPU, and its host controller matches the
+oracle bit for bit."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2305_12213_b200 import binding, inputs
+from paper_2305_12213_b200 import build as dbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    dbuild.build()
+    return binding.lib()
+
+
+def _declared_symbols():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for fn in os.listdir(inc):
+        text = open(os.path.join(inc, fn)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names.update(re.findall(r"\b(db_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
+
+
+def test_header_symbols_are_exported(lib):
+    names = _declared_symbols()
+    assert "db_aggregate_update" in names and "db_worker_grad" in names and "db_controller_step" in names
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in include/ but not exported"
+
+
+def test_binding_covers_every_symbol(lib):
+    assert sorted(binding._SIGNATURES) == _declared_symbols()
+
+
+def test_status_strings(lib):
+    assert lib.db_status_string(0) == b"ok"
+    assert len({lib.db_status_string(i) for i in range(6)}) == 6
+    assert lib.db_last_cuda_error() is not None
+
+
+def test_workspace_queries(lib):
+    assert lib.db_aggregate_workspace_bytes(8, 1 << 20) >= 256 + 8 * 148
+    assert lib.db_worker_grad_workspace_bytes(24, 2048, 1000) >= 4 * 24 * 1000 * 2
+    assert lib.db_worker_grad_workspace_bytes(0, 2048, 1000) == 0
+
+
+def _agg(lib, grads, b, K, N, p=0x1000, v=0x2000000, lr=0.1, mu=0.9, dtype=0, sq=None, ws=None, wsb=0):
+    table = (ctypes.c_void_p * max(1, len(grads)))(*grads) if grads is not None else None
+    bb = (ctypes.c_int32 * max(1, len(b)))(*b) if b is not None else None
+    return lib.db_aggregate_update_ex(
+        None if table is None else ctypes.cast(table, ctypes.c_void_p), dtype,
+        None if bb is None else ctypes.cast(bb, ctypes.c_void_p), K, N, p, v, lr, mu, sq, ws, wsb, None)
+
+
+def test_aggregate_argument_validation_never_reaches_the_gpu(lib):
+    g = [0x40000000, 0x50000000]
+    E = binding
+    assert _agg(lib, None, [1, 1], 2, 16) == E.DB_ERR_NULL
+    assert _agg(lib, g, None, 2, 16) == E.DB_ERR_NULL
+    assert _agg(lib, g, [1, 1], 0, 16) == E.DB_ERR_ARG
+    assert _agg(lib, g, [1, 1], E.DB_MAX_K + 1, 16) == E.DB_ERR_ARG
+    assert _agg(lib, g, [1, 1], 2, -1) == E.DB_ERR_ARG
+    assert _agg(lib, g, [1, -1], 2, 16) == E.DB_ERR_ARG
+    assert _agg(lib, g, [0, 0], 2, 16) == E.DB_ERR_ARG
+    assert _agg(lib, g, [1, 1], 2, 16, lr=float("nan")) == E.DB_ERR_ARG
+    assert _agg(lib, g, [1, 1], 2, 16, mu=float("inf")) == E.DB_ERR_ARG
+    assert _agg(lib, g, [1, 1], 2, 16, dtype=7) == E.DB_ERR_UNSUPPORTED
+    assert _agg(lib, g, [1, 1], 2, 16, p=None) == E.DB_ERR_NULL
+    assert _agg(lib, [0x40000000, None], [1, 1], 2, 16) == E.DB_ERR_NULL
+    # N == 0 is fine and enqueues nothing
+    assert _agg(lib, g, [1, 1], 2, 0) == E.DB_OK
+    # overlapping buffers
+    assert _agg(lib, g, [1, 1], 2, 1024, p=0x1000, v=0x1800) == E.DB_ERR_ARG
+    assert _agg(lib, [0x1100, 0x50000000], [1, 1], 2, 1024, p=0x1000) == E.DB_ERR_ARG
+    # a zero-batch worker's pointer is ignored entirely, even NULL or overlapping
+    assert _agg(lib, [None, 0x50000000], [0, 1], 2, 0) == E.DB_OK
+    # norm requested without a workspace
+    assert _agg(lib, g, [1, 1], 2, 16, sq=0x3000) == E.DB_ERR_NULL
+    assert _agg(lib, g, [1, 1], 2, 16, sq=0x3000, ws=0x7000, wsb=8) == E.DB_ERR_ARG
+    # misaligned element pointers
+    assert _agg(lib, [0x40000002, 0x50000000], [1, 1], 2, 16) == E.DB_ERR_ARG
+
+
+def test_worker_grad_argument_validation(lib):
+    E = binding
+    f = lib.db_worker_grad
+    ok = dict(X=0x1000, y=0x2000, W=0x3000, b=4, D=8, C=8, G=0x4000, loss=None, ws=0x8000, wsb=1 << 20)
+
+    def call(**kw):
+        a = dict(ok, **kw)
+        return f(a["X"], a["y"], a["W"], a["b"], a["D"], a["C"], a["G"], a["loss"], a["ws"], a["wsb"], None)
+
+    assert call(X=None) == E.DB_ERR_NULL
+    assert call(G=None) == E.DB_ERR_NULL
+    assert call(ws=None) == E.DB_ERR_NULL
+    assert call(b=0) == E.DB_ERR_ARG
+    assert call(b=70000) == E.DB_ERR_ARG
+    assert call(D=0) == E.DB_ERR_ARG
+    assert call(wsb=16) == E.DB_ERR_ARG
+    assert call(ws=0x8004) == E.DB_ERR_ARG
+
+
+# ------------------------------------------------------------------ host controller vs oracle
+def test_controller_fixed_point_and_paper_rule(lib):
+    assert binding.controller_step([16, 32, 80], [1.0, 2.0, 5.0], 0.5) == [16, 32, 80]
+    assert binding.controller_step([32] * 8, [10.0] * 4 + [1.0] * 4, 1.0) == [58] * 4 + [6] * 4
+
+
+@pytest.mark.parametrize("seed", range(200))
+def test_controller_bit_exact_against_oracle(lib, seed):
+    rng = np.random.default_rng(seed)
+    K = int(rng.integers(1, 33))
+    b = inputs.batch_sizes_uniform(K, 0 if seed % 5 == 0 else 8, 256, seed)
+    if sum(b) == 0:
+        b[0] = 3
+    X = inputs.lognormal_throughputs(K, 0.5 + (seed % 3), seed + 7)
+    kp = float(rng.choice([0.1, 0.5, 0.9, 1.0]))
+    S = sum(b)
+    lo = hi = None
+    if seed % 4 == 1:
+        lo = [int(x) for x in rng.integers(0, max(1, S // (2 * K)) + 1, size=K)]
+    if seed % 4 == 2:
+        hi = [int(x) for x in rng.integers(S // K + 1, S + 2, size=K)]
+    traj_lib, traj_ref = list(b), np.array(b, dtype=np.int32)
+    for _ in range(6):
+        try:
+            ref = oracle.controller_step(traj_ref, X, kp, lo, hi)
+        except oracle.OracleError as e:
+            with pytest.raises(binding.DynbatchError) as ei:
+                binding.controller_step(traj_lib, X, kp, lo, hi)
+            assert ei.value.status == e.code
+            return
+        got = binding.controller_step(traj_lib, X, kp, lo, hi)
+        assert got == ref.tolist()
+        assert sum(got) == S
+        traj_lib, traj_ref = got, ref
+
+
+def test_controller_rejects_bad_arguments(lib):
+    E = binding
+    for X in ([1.0, 0.0], [1.0, -1.0], [1.0, float("nan")], [float("inf"), 1.0]):
+        with pytest.raises(E.DynbatchError) as ei:
+            E.controller_step([4, 4], X, 1.0)
+        assert ei.value.status == E.DB_ERR_ARG
+    for kp in (0.0, -1.0, 1.0001, float("nan")):
+        with pytest.raises(E.DynbatchError):
+            E.controller_step([4, 4], [1.0, 2.0], kp)
+    with pytest.raises(E.DynbatchError) as ei:
+        E.controller_step([4, 4], [1.0, 2.0], 1.0, b_min=[5, 5])
+    assert ei.value.status == E.DB_ERR_INFEASIBLE
+    with pytest.raises(E.DynbatchError) as ei:
+        E.controller_step([4, 4], [1.0, 2.0], 1.0, b_max=[3, 3])
+    assert ei.value.status == E.DB_ERR_INFEASIBLE
+    assert lib.db_controller_step(None, None, 2, 1.0) == E.DB_ERR_NULL
+
+
+def test_controller_scenario_with_throughput_drop(lib):
+    """16 lognormal workers, one halves its throughput mid-run: both sides track it identically."""
+    X = inputs.lognormal_throughputs(16, 0.5, 4242)
+    b_lib, b_ref = [32] * 16, np.full(16, 32, dtype=np.int32)
+    for it in range(200):
+        if it == 50:
+            X[3] *= 0.5
+        b_ref = oracle.controller_step(b_ref, X, 1.0)
+        b_lib = binding.controller_step(b_lib, X, 1.0)
+        assert b_lib == b_ref.tolist() and sum(b_lib) == 512
+    want = 512 * np.array(X) / sum(X)
+    assert np.abs(np.array(b_lib) - want).max() <= 1.0

@@ -1,0 +1,76 @@
+"""GPU parity of db_worker_grad against the fp64 oracle, and the closed-form check that the
+batch-weighted aggregate of per-worker gradients is the gradient of the concatenated batch."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import FP32_TOL, f64, rel_err
+from paper_2305_12213_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _worker_grad(X, y, W):
+    b_i, D = X.shape
+    C = W.shape[1]
+    G = torch.empty(D, C, device=DEV)
+    loss = torch.zeros(1, device=DEV)
+    ws = torch.empty(binding.worker_grad_workspace_bytes(b_i, D, C), dtype=torch.uint8, device=DEV)
+    binding.worker_grad(X, y, W, G, loss, ws)
+    torch.cuda.synchronize()
+    return G, float(loss.item())
+
+
+@pytest.mark.parametrize("b_i,D,C", [(1, 4, 4), (5, 6, 3), (7, 33, 10), (24, 128, 64), (3, 257, 130),
+                                      (65, 200, 96), (130, 64, 1000), (40, 2048, 1000)])
+def test_shapes_including_ragged_tiles(b_i, D, C):
+    X, y, W = inputs.softmax_problem([b_i], D, C, seed=100 + b_i, w_std=0.05, device=DEV)
+    G, loss = _worker_grad(X, y, W)
+    rG, rloss = oracle.worker_grad(X.cpu().numpy(), y.cpu().numpy(), W.cpu().numpy())
+    assert rel_err(f64(G), rG) <= FP32_TOL
+    assert abs(loss - rloss) <= FP32_TOL * abs(rloss)
+    assert float(G.double().sum(dim=1).abs().max()) < 1e-5      # rows of P - Y sum to zero
+
+
+def test_out_of_range_label_contributes_no_onehot():
+    X, y, W = inputs.softmax_problem([4], 16, 8, seed=7, w_std=0.1, device=DEV)
+    y2 = y.clone()
+    y2[1] = 99
+    G, _ = _worker_grad(X, y2, W)
+    # the row sums of P alone are 1: column-sum identity is broken exactly by sample 1's features
+    excess = G.double().sum(dim=1) * 4
+    assert rel_err(excess.cpu().numpy(), f64(X[1])) <= 1e-5
+
+
+def test_config_ragged_four_workers_against_the_concatenated_batch():
+    """D=2048, C=1000, b={24,40,64,128}: per-worker gradients, then the weighted aggregate,
+    which must be the mean gradient of all 256 samples."""
+    bs = [24, 40, 64, 128]
+    D, C = 2048, 1000
+    X, y, W = inputs.softmax_problem(bs, D, C, seed=3000, device=DEV)
+    offs = np.concatenate([[0], np.cumsum(bs)])
+    Xh, yh, Wh = X.cpu().numpy(), y.cpu().numpy(), W.cpu().numpy()
+    Gs = []
+    for i, b_i in enumerate(bs):
+        s, e = int(offs[i]), int(offs[i + 1])
+        G, loss = _worker_grad(X[s:e].contiguous(), y[s:e].contiguous(), W)
+        rG, rloss = oracle.worker_grad(Xh[s:e], yh[s:e], Wh)
+        assert rel_err(f64(G), rG) <= FP32_TOL, f"worker {i}"
+        assert abs(loss - rloss) <= FP32_TOL * abs(rloss)
+        Gs.append(G.reshape(-1))
+    N = D * C
+    p, v = torch.zeros(N, device=DEV), torch.zeros(N, device=DEV)
+    sq = torch.zeros(1, dtype=torch.float64, device=DEV)
+    ws = torch.empty(binding.aggregate_workspace_bytes(4, N), dtype=torch.uint8, device=DEV)
+    binding.aggregate_update(Gs, bs, p, v, 1.0, 0.0, sq, ws)      # p = -aggregate, v = aggregate
+    torch.cuda.synchronize()
+    full, _ = oracle.worker_grad(Xh, yh, Wh)                       # all 256 rows, divisor 256
+    full = full.reshape(-1)
+    assert rel_err(f64(v), full) <= FP32_TOL
+    assert rel_err(f64(p), -full) <= FP32_TOL
+    assert abs(float(sq.item()) - float(full @ full)) <= FP32_TOL * float(full @ full)
+    # the uniform average of the four gradients is a different vector
+    uniform = torch.stack(Gs).double().mean(0).cpu().numpy()
+    assert rel_err(uniform, full) > 1e-2
