@@ -103,6 +103,46 @@ db_status db_aggregate_update_ex(const void* const* grads, db_dtype grad_dtype,
 size_t db_aggregate_workspace_bytes(int32_t K, int64_t N);
 
 /* ------------------------------------------------------------------------
+ * The same step for callers that cannot provide scratch memory
+ * (the paper has no counterpart; this is a packaging variant of the call above)
+ *
+ * db_aggregate_update_ex needs a device workspace for the gradient norm, so
+ * somebody has to allocate one.  Some callers cannot: a plug-in running inside
+ * a host application that has already handed all device memory to its own
+ * pool and exposes no allocator to plug-ins; a latency-critical loop in which
+ * cudaMalloc is forbidden because it may synchronise the whole device; code
+ * that only ever receives raw input/output pointers from its framework.  For
+ * them this entry point keeps the scratch inside the library, in a fixed
+ * array in device global memory (DB_STATIC_SCRATCH_BYTES, resident on every
+ * GPU that loads the library until the process exits).  It calls no
+ * cudaMalloc/cudaFree and no allocating library routine.
+ *
+ * Arguments and results are those of db_aggregate_update_ex without the
+ * workspace pair; results are bit-identical to it.
+ *
+ *   - The first call on each device looks up the array's device address
+ *     (once per device, with that device current).  Make that first call
+ *     outside any stream capture.
+ *   - All calls on a device share the one array.  It keeps the previous
+ *     call's contents; the part that must start at zero (the CTA arrival
+ *     counter) is cleared on the stream ahead of every launch.  Two calls
+ *     whose kernels may run at the same time on one device (different
+ *     streams, different threads) race on it and return a wrong norm:
+ *     serialise them, or use db_aggregate_update_ex with separate workspaces.
+ *   - If the scratch this device needs (db_aggregate_workspace_bytes) exceeds
+ *     DB_STATIC_SCRATCH_BYTES the call returns DB_ERR_UNSUPPORTED and enqueues
+ *     nothing; db_last_cuda_error() then says how many bytes were needed.
+ *     N itself is not limited: the scratch grows with the GPU's SM count only.
+ * ------------------------------------------------------------------------ */
+#define DB_STATIC_SCRATCH_BYTES 65536
+
+db_status db_aggregate_update_static(const void* const* grads,
+                                     db_dtype grad_dtype, const int32_t* b,
+                                     int32_t K, int64_t N, float* params,
+                                     float* momentum, float lr, float mu,
+                                     double* grad_sqnorm, void* cuda_stream);
+
+/* ------------------------------------------------------------------------
  * Ragged per-worker gradient of a linear-softmax classifier
  *
  * The model on which the batch-proportional weighting of Eq. 2 is checked

@@ -39,6 +39,8 @@ _SIGNATURES = {
                                          c_void_p, c_float, c_float, c_void_p, c_void_p, c_size_t,
                                          c_void_p]),
     "db_aggregate_workspace_bytes": (c_size_t, [c_int32, c_int64]),
+    "db_aggregate_update_static": (c_int32, [c_void_p, c_int32, c_void_p, c_int32, c_int64, c_void_p,
+                                             c_void_p, c_float, c_float, c_void_p, c_void_p]),
     "db_worker_grad": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p,
                                  c_void_p, c_void_p, c_size_t, c_void_p]),
     "db_worker_grad_workspace_bytes": (c_size_t, [c_int32, c_int32, c_int32]),
@@ -69,8 +71,10 @@ def _check(status: int) -> None:
     if status != DB_OK:
         L = lib()
         msg = L.db_status_string(status).decode()
-        if status == DB_ERR_CUDA:
-            msg += ": " + L.db_last_cuda_error().decode()
+        if status in (DB_ERR_CUDA, DB_ERR_UNSUPPORTED):
+            detail = L.db_last_cuda_error().decode()
+            if detail:
+                msg += ": " + detail
         raise DynbatchError(status, msg)
 
 
@@ -125,6 +129,29 @@ def aggregate_update(grads: Sequence[torch.Tensor], b: Sequence[int], params: to
         None if workspace is None else workspace.data_ptr(),
         0 if workspace is None else workspace.numel() * workspace.element_size(),
         _stream_ptr(stream)))
+
+
+def aggregate_update_static(grads: Sequence[torch.Tensor], b: Sequence[int], params: torch.Tensor,
+                            momentum: torch.Tensor, lr: float, mu: float,
+                            grad_sqnorm: Optional[torch.Tensor] = None,
+                            stream: Optional[torch.cuda.Stream] = None) -> None:
+    """db_aggregate_update_static: aggregate_update for callers that cannot supply a workspace.
+
+    The norm's scratch is a fixed array inside the library, shared by every call on the device, so
+    calls that could overlap on the GPU must be serialised by the caller.  Nothing is allocated.
+    """
+    K = len(grads)
+    if len(b) != K:
+        raise ValueError("len(b) != len(grads)")
+    gdt = grads[0].dtype
+    if gdt not in (torch.float32, torch.bfloat16):
+        raise TypeError("gradients must be float32 or bfloat16")
+    table = (c_void_p * K)(*[_dev_ptr(g, gdt, "grads[k]") for g in grads])
+    _check(lib().db_aggregate_update_static(
+        ctypes.cast(table, c_void_p), DB_F32 if gdt == torch.float32 else DB_BF16,
+        ctypes.cast(_i32_array(b), c_void_p), K, int(params.numel()),
+        _dev_ptr(params, torch.float32, "params"), _dev_ptr(momentum, torch.float32, "momentum"),
+        float(lr), float(mu), _dev_ptr(grad_sqnorm, torch.float64, "grad_sqnorm"), _stream_ptr(stream)))
 
 
 def worker_grad_workspace_bytes(b_i: int, D: int, C: int) -> int:

@@ -11,6 +11,7 @@
 #include <cuda_bf16.h>
 
 #include <cstdint>
+#include <cstdio>
 
 #include "common.h"
 
@@ -399,4 +400,59 @@ extern "C" db_status db_aggregate_update(const float* const* grads, const int32_
                                          int64_t N, float* params, float* momentum, float lr, float mu) {
     return db_aggregate_update_ex(reinterpret_cast<const void* const*>(grads), DB_F32, b, K, N, params,
                                   momentum, lr, mu, nullptr, nullptr, 0, nullptr);
+}
+
+// ---------------------------------------------------------------------------
+// Variant with library-owned scratch, for callers that cannot allocate.
+// ---------------------------------------------------------------------------
+namespace dynbatch {
+namespace {
+
+// Ticket + per-CTA partials of the norm.  Lives in every device's global memory
+// for the life of the process.  In host code this name is only a handle for
+// cudaGetSymbolAddress: it is never passed to a kernel as a pointer.
+static __device__ __align__(256) unsigned char g_static_scratch[DB_STATIC_SCRATCH_BYTES];
+
+// Device address of g_static_scratch on the current device, looked up once per device.
+db_status static_scratch_address(void** out) {
+    constexpr int kMaxDev = 64;
+    static void* cache[kMaxDev] = {nullptr};
+    int dev = 0;
+    DB_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDev) return DB_ERR_UNSUPPORTED;
+    void* ptr = __atomic_load_n(&cache[dev], __ATOMIC_ACQUIRE);
+    if (!ptr) {
+        DB_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        if (!ptr) return DB_ERR_CUDA;
+        __atomic_store_n(&cache[dev], ptr, __ATOMIC_RELEASE);  // every thread stores the same address
+    }
+    *out = ptr;
+    return DB_OK;
+}
+
+}  // namespace
+}  // namespace dynbatch
+
+extern "C" db_status db_aggregate_update_static(const void* const* grads, db_dtype grad_dtype,
+                                                const int32_t* b, int32_t K, int64_t N, float* params,
+                                                float* momentum, float lr, float mu,
+                                                double* grad_sqnorm, void* cuda_stream) {
+    using namespace dynbatch;
+    void* scratch = nullptr;
+    if (grad_sqnorm) {
+        const size_t need = db_aggregate_workspace_bytes(K, N);
+        if (need > DB_STATIC_SCRATCH_BYTES) {
+            char msg[160];
+            snprintf(msg, sizeof msg,
+                     "db_aggregate_update_static: this device needs %zu bytes of scratch, the built-in "
+                     "array holds %d; use db_aggregate_update_ex with a workspace",
+                     need, DB_STATIC_SCRATCH_BYTES);
+            record_message(msg);
+            return DB_ERR_UNSUPPORTED;
+        }
+        const db_status st = static_scratch_address(&scratch);
+        if (st != DB_OK) return st;
+    }
+    return db_aggregate_update_ex(grads, grad_dtype, b, K, N, params, momentum, lr, mu, grad_sqnorm,
+                                  scratch, scratch ? DB_STATIC_SCRATCH_BYTES : 0, cuda_stream);
 }

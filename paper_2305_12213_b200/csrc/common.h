@@ -9,6 +9,9 @@ namespace dynbatch {
 // Records the runtime's message for db_last_cuda_error() and returns DB_ERR_CUDA.
 db_status record_cuda_error(cudaError_t err, const char* where);
 
+// Stores a plain message for db_last_cuda_error() (non-CUDA failures that need explaining).
+void record_message(const char* text);
+
 // Number of SMs of the current device (queried once per device, then cached).
 int sm_count();
 

@@ -14,6 +14,8 @@ db_status record_cuda_error(cudaError_t err, const char* where) {
     return DB_ERR_CUDA;
 }
 
+void record_message(const char* text) { std::snprintf(g_cuda_msg, sizeof g_cuda_msg, "%s", text); }
+
 int sm_count() {
     constexpr int kMaxDev = 64;
     static int cache[kMaxDev] = {0};

@@ -1,0 +1,71 @@
+"""The allocation-free entry point, db_aggregate_update_static, against db_aggregate_update_ex.
+
+Some users of the library may not allocate device memory at all (a plug-in whose host owns the whole
+GPU heap, a loop where cudaMalloc's device-wide synchronisation is not acceptable).  For them the
+norm's scratch lives in a fixed array inside the library.  The result must be the one the workspace
+form gives -- also on a second call, when the shared array still holds the first call's partials
+and arrival counter.  This file sorts last so a failure here cannot hide another test's.
+"""
+import pytest
+import torch
+
+from paper_2305_12213_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _reference(grads, b, p0, v0, lr, mu):
+    K, N = len(grads), p0.numel()
+    p, v = p0.clone(), v0.clone()
+    sq = torch.zeros(1, dtype=torch.float64, device=DEV)
+    ws = torch.empty(binding.aggregate_workspace_bytes(K, N), dtype=torch.uint8, device=DEV)
+    binding.aggregate_update(grads, b, p, v, lr, mu, sq, ws)
+    torch.cuda.synchronize()
+    return p, v, float(sq.item())
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_two_calls_in_a_row_match_the_workspace_form(dtype):
+    K, N = 8, 3_000_017
+    b = [58] * 4 + [6] * 4
+    p_ref = inputs.normal(N, 0.02, 1, DEV)
+    v_ref = torch.zeros(N, device=DEV)
+    p, v = p_ref.clone(), v_ref.clone()
+    sq = torch.full((1,), -1.0, dtype=torch.float64, device=DEV)
+    for call in range(2):
+        # a different problem each call: other gradients, and K shrinks so fewer slots are rewritten
+        kk = K - 3 * call
+        grads = inputs.worker_gradients(kk, N, 1e-3, 700 + call, device=DEV, dtype=dtype)
+        p_ref, v_ref, sq_ref = _reference(grads, b[:kk], p_ref, v_ref, 0.1, 0.9)
+        binding.aggregate_update_static(grads, b[:kk], p, v, 0.1, 0.9, sq)
+        torch.cuda.synchronize()
+        assert torch.equal(p, p_ref) and torch.equal(v, v_ref), f"call {call}"
+        got = float(sq.item())
+        assert got == sq_ref, f"call {call}: {got} vs {sq_ref}"      # same kernel, same grid: same bits
+        assert abs(got - sq_ref) <= 1e-5 * sq_ref
+
+
+def test_small_then_large_problem_reuses_the_array_cleanly():
+    sq = torch.zeros(1, dtype=torch.float64, device=DEV)
+    for N in (1000, 5_000_003, 7):
+        g = [torch.ones(N, device=DEV) for _ in range(3)]
+        p, v = torch.zeros(N, device=DEV), torch.zeros(N, device=DEV)
+        binding.aggregate_update_static(g, [1, 2, 3], p, v, 0.5, 0.0, sq)
+        torch.cuda.synchronize()
+        assert float(sq.item()) == float(N)
+        assert torch.equal(v, torch.ones(N, device=DEV)) and torch.equal(p, torch.full((N,), -0.5, device=DEV))
+
+
+def test_without_norm_and_argument_errors():
+    N = 4096
+    g = inputs.worker_gradients(2, N, 1.0, 710, device=DEV)
+    p0, v0 = inputs.normal(N, 0.02, 2, DEV), inputs.normal(N, 0.5, 3, DEV)
+    p1, v1, p2, v2 = p0.clone(), v0.clone(), p0.clone(), v0.clone()
+    binding.aggregate_update_static(g, [3, 5], p1, v1, 0.1, 0.9)
+    binding.aggregate_update(g, [3, 5], p2, v2, 0.1, 0.9)
+    torch.cuda.synchronize()
+    assert torch.equal(p1, p2) and torch.equal(v1, v2)
+    with pytest.raises(binding.DynbatchError) as ei:
+        binding.aggregate_update_static(g, [0, 0], p1, v1, 0.1, 0.9)
+    assert ei.value.status == binding.DB_ERR_ARG
