@@ -2,6 +2,7 @@
 """Benchmark of the fused parameter-server step (weighted aggregation + momentum SGD).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload resnet50|bert_base|small|sweep]
 
 One step = one pass of the hot path over one batch of synthetic input: the host
 controller chooses the batch sizes, then db_aggregate_update_ex combines the K
@@ -33,19 +34,64 @@ import torch
 from paper_2305_12213_b200 import inputs, replicas
 
 METRIC = "aggregate+update HBM GB/s (% of B200 peak) and iterations/s at ResNet-50 size"
-WORKLOAD = "resnet50_arena_N25557032_K8_fp32_gbatch256"
-K_WORKERS = 8
-N_PARAMS = inputs.RESNET50_N
-THROUGHPUTS = [10.0] * 4 + [1.0] * 4
-B0 = [32] * 8
-KP, LR, MU = 1.0, 0.1, 0.9
-GRAD_STD, PARAM_STD = 1e-3, 0.02
 FALLBACK_HBM_GBS = 6650.0
+L2_BYTES = 126 * 1024 * 1024
+PARAM_STD = 0.02
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the aggregation kernel on this
-# workload, from the ncu capture summarised under profiles/, with the digest of the kernel source
-# the counters belong to.  Reported as null once the source has changed.
-NCU_TRAFFIC = {"bytes_per_launch": 1200815616,
+
+class Workload:
+    """One synthetic configuration of the step: K workers, N parameters, gradient dtype, controller inputs."""
+
+    def __init__(self, name, K, N, grad_dtype, b0, throughputs, kp, lr, mu, grad_std):
+        self.name, self.K, self.N, self.grad_dtype = name, K, N, grad_dtype
+        self.b0, self.throughputs, self.kp, self.lr, self.mu, self.grad_std = b0, throughputs, kp, lr, mu, grad_std
+
+    @property
+    def grad_bytes(self):
+        return 2 if self.grad_dtype == torch.bfloat16 else 4
+
+    @property
+    def bytes_per_step(self):
+        return step_bytes(self.K, self.N, self.grad_bytes)
+
+    @property
+    def working_set(self):
+        return self.K * self.N * self.grad_bytes + 2 * self.N * 4
+
+
+def resnet50_workload():
+    return Workload("resnet50_arena_N25557032_K8_fp32_gbatch256", 8, inputs.RESNET50_N, torch.float32,
+                    [32] * 8, [10.0] * 4 + [1.0] * 4, 1.0, 0.1, 0.9, 1e-3)
+
+
+def bert_base_workload():
+    return Workload("bert_base_arena_N109482240_K16_bf16_gbatch512", 16, inputs.BERT_BASE_N, torch.bfloat16,
+                    [32] * 16, inputs.lognormal_throughputs(16, 0.5, 4242), 1.0, 0.05, 0.9, 1e-3)
+
+
+def small_workload():
+    return Workload("small_N1048576_K3_fp32_gbatch128", 3, 1 << 20, torch.float32, [16, 32, 80],
+                    [1.0, 2.0, 5.0], 0.5, 0.1, 0.9, 1.0)
+
+
+def sweep_workloads():
+    out = []
+    for n in (1 << 20, 1 << 22, 1 << 24, 1 << 26, 1 << 28):
+        for k in (2, 4, 8, 16, 32):
+            if n * k <= (1 << 33):
+                b = inputs.batch_sizes_uniform(k, 8, 256, 5000 + k)
+                # throughputs proportional to b: the controller step runs and holds b fixed
+                out.append(Workload(f"sweep_N{n}_K{k}_fp32", k, n, torch.float32, b, [float(x) for x in b],
+                                    1.0, 0.1, 0.9, 1.0))
+    return out
+
+
+WORKLOADS = {"resnet50": resnet50_workload, "bert_base": bert_base_workload, "small": small_workload}
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the aggregation kernel on the
+# resnet50 workload, from the ncu capture summarised under profiles/, with the digest of the kernel
+# source the counters belong to.  Reported as null once the source has changed.
+NCU_TRAFFIC = {"workload": "resnet50_arena_N25557032_K8_fp32_gbatch256", "bytes_per_launch": 1200815616,
                "aggregate_cu_sha256": "a3bd1b313e6fbb98af38dea48f0e81ad2610b5b27e756cf20fc5ff0f69c4c2dc"}
 
 
@@ -63,7 +109,9 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def kernel_traffic():
+def kernel_traffic(workload_name):
+    if workload_name != NCU_TRAFFIC["workload"]:
+        return None
     src = os.path.join(ROOT, "paper_2305_12213_b200", "csrc", "aggregate.cu")
     try:
         digest = hashlib.sha256(open(src, "rb").read()).hexdigest()
@@ -130,73 +178,119 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------------------------
-def run_ours(args):
-    from paper_2305_12213_b200 import binding, build
-    rank, local_rank, world = replicas.env_world()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device; libdynbatch has no CPU fallback")
-    dev = torch.device("cuda", local_rank if world > 1 else 0)
-    torch.cuda.set_device(dev)
-    replicas.init(device=dev)
-    if rank == 0:
-        build.build()
-    replicas.barrier(dev)
-    binding.lib()
-
-    K, N = K_WORKERS, N_PARAMS
+def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
+    """Times `args.steps` steps of workload `wl` on `dev`; returns the JSON record (all ranks)."""
+    from paper_2305_12213_b200 import binding
+    K, N = wl.K, wl.N
     seed = 2000 + 17 * rank
-    grads = inputs.worker_gradients(K, N, GRAD_STD, seed, device=dev)
+    grads = inputs.worker_gradients(K, N, wl.grad_std, seed, device=dev, dtype=wl.grad_dtype)
     p = inputs.normal(N, PARAM_STD, seed + 500, dev)
     v = torch.zeros(N, device=dev)
     sq = torch.zeros(1, dtype=torch.float64, device=dev)
     ws = torch.empty(binding.aggregate_workspace_bytes(K, N), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
-    b = list(B0)
+    b = list(wl.b0)
+    # inputs smaller than twice the L2 would be served from it on the next step: flush in between
+    flush = None
+    if wl.working_set < 2 * L2_BYTES:
+        flush = torch.empty(2 * L2_BYTES // 4, dtype=torch.int32, device=dev)
 
     def step():
         nonlocal b
-        b = binding.controller_step(b, THROUGHPUTS, KP)
-        binding.aggregate_update(grads, b, p, v, LR, MU, sq, ws, stream)
+        b = binding.controller_step(b, wl.throughputs, wl.kp)
+        binding.aggregate_update(grads, b, p, v, wl.lr, wl.mu, sq, ws, stream)
 
-    for _ in range(max(3, args.warmup)):
+    warmup = max(3, args.warmup)
+    for _ in range(warmup):
         step()
     torch.cuda.synchronize()
 
     # ---- timed region: device-resident inputs
-    events = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    steps = args.steps
     sampler = ClockSampler(dev.index)
     replicas.barrier(dev)
     torch.cuda.synchronize()
-    with sampler:
-        for i in range(args.steps):
-            events[i].record(stream)
-            step()
-        events[args.steps].record(stream)
-        torch.cuda.synchronize()
+    if flush is None:
+        events = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        with sampler:
+            for i in range(steps):
+                events[i].record(stream)
+                step()
+            events[steps].record(stream)
+            torch.cuda.synchronize()
+        per_step_ms = [events[i].elapsed_time(events[i + 1]) for i in range(steps)]
+        elapsed_ms = events[0].elapsed_time(events[steps])
+    else:
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        with sampler:
+            for e0, e1 in pairs:
+                # write 252 MB (evicts the step's lines), then read it back so that the L2 is left
+                # holding clean lines and the timed kernel does not pay for their write-back
+                flush.fill_(1)
+                flush.sum()
+                e0.record(stream)
+                step()
+                e1.record(stream)
+            torch.cuda.synchronize()
+        per_step_ms = [e0.elapsed_time(e1) for e0, e1 in pairs]
+        elapsed_ms = float(np.sum(per_step_ms))
     replicas.barrier(dev)
-    elapsed_ms = events[0].elapsed_time(events[args.steps])
-    per_step_ms = [events[i].elapsed_time(events[i + 1]) for i in range(args.steps)]
-    bytes_step = step_bytes(K, N, 4)
-    job_bps, max_ms = replicas.job_throughput(bytes_step * args.steps, elapsed_ms, dev)
+    bytes_step = wl.bytes_per_step
+    job_bps, max_ms = replicas.job_throughput(bytes_step * steps, elapsed_ms, dev)
     final_sq = float(sq.item())
     assert np.isfinite(final_sq) and final_sq > 0 and bool(torch.isfinite(p[:1024]).all())
 
-    # ---- end to end: gradients arrive in pinned host memory, parameters go back to the host
+    peak, peak_kind = measured_peak()
+    kernel_ms = float(np.mean(per_step_ms))
+    achieved = bytes_step / (kernel_ms * 1e-3) / 1e9
+    gname = "float" if wl.grad_dtype == torch.float32 else "__nv_bfloat16"
+    out = {
+        "metric": METRIC, "value": job_bps / 1e9, "unit": "GB/s",
+        "iterations_per_s": world * steps / (max_ms * 1e-3),
+        "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": max_ms / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "K": K, "N": N,
+                   "grad_dtype": "f32" if wl.grad_dtype == torch.float32 else "bf16",
+                   "global_batch": sum(wl.b0), "kp": wl.kp, "lr": wl.lr, "mu": wl.mu, "grad_sqnorm": True,
+                   "bytes_per_step": bytes_step,
+                   "l2": ("inputs (%.2f GB per step) exceed the 126 MB L2" % (wl.working_set / 1e9)) if flush is None
+                   else "L2 flushed (252 MB written, then read) before every timed step",
+                   "parallelism": f"{world} independent replica(s), no collective"},
+        "gpu_launches": steps,
+        "clocks": sampler.summary(),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_source": f"of {peak_kind}",
+                     "kernel": f"agg_vec_kernel<{gname}, {K if K <= 16 else 0}, *, true>", "kernel_ms": kernel_ms,
+                     "kernel_ms_min": float(np.min(per_step_ms)), "traffic": kernel_traffic(wl.name)},
+    }
+    if with_e2e:
+        out["e2e"] = measure_e2e(wl, args, dev, grads, p, v, b)
+    if with_cpu and rank == 0 and world == 1:
+        out["cpu_baseline"] = cpu_baseline(wl, host_gradients(grads), b)
+    return out
+
+
+def measure_e2e(wl, args, dev, grads, p, v, b):
+    """The same step through db_aggregate_update_host: the gradients are in pinned host memory, the
+    updated parameters and the norm come back to the host; all copies are inside the timed region."""
+    from paper_2305_12213_b200 import binding
+    K, N = wl.K, wl.N
+    stream = torch.cuda.current_stream()
     e2e_steps = max(3, min(args.steps, 20))
-    host_grads = [torch.empty(N, dtype=torch.float32).pin_memory() for _ in range(K)]
+    host_grads = [torch.empty(N, dtype=wl.grad_dtype).pin_memory() for _ in range(K)]
     for hg, g in zip(host_grads, grads):
         hg.copy_(g)
     host_p = torch.empty(N, dtype=torch.float32).pin_memory()
-    host_sq = torch.empty(1, dtype=torch.float64).pin_memory()
+    host_sq = torch.zeros(1, dtype=torch.float64).pin_memory()
+    pipe = binding.HostPipeline()
+    staging = torch.empty(binding.host_staging_bytes(K, wl.grad_dtype, N, 0), dtype=torch.uint8, device=dev)
+    b = list(b)
 
     def e2e_step():
         nonlocal b
-        for hg, g in zip(host_grads, grads):
-            g.copy_(hg, non_blocking=True)
-        b = binding.controller_step(b, THROUGHPUTS, KP)
-        binding.aggregate_update(grads, b, p, v, LR, MU, sq, ws, stream)
-        host_p.copy_(p, non_blocking=True)
-        host_sq.copy_(sq, non_blocking=True)
+        b = binding.controller_step(b, wl.throughputs, wl.kp)
+        pipe.aggregate_update(host_grads, b, p, v, wl.lr, wl.mu, host_p, host_sq, staging, 0, stream)
         stream.synchronize()          # the step's result is on the host before the next one starts
 
     for _ in range(2):
@@ -211,56 +305,66 @@ def run_ours(args):
     torch.cuda.synchronize()
     replicas.barrier(dev)
     e2e_ms = e0.elapsed_time(e1)
-    e2e_bps, _ = replicas.job_throughput(bytes_step * e2e_steps, e2e_ms, dev)
+    assert np.isfinite(float(host_sq[0])) and float(host_sq[0]) > 0 and bool(torch.isfinite(host_p[:1024]).all())
+    e2e_bps, e2e_max_ms = replicas.job_throughput(wl.bytes_per_step * e2e_steps, e2e_ms, dev)
+    nchunks = -(-N // (1 << 21))
+    pipe.close()
+    return {"value": e2e_bps / 1e9, "unit": "GB/s", "steps": e2e_steps, "ms_per_step": e2e_max_ms / e2e_steps,
+            "h2d_bytes_per_step": K * N * wl.grad_bytes, "d2h_bytes_per_step": N * 4 + 8,
+            "api": "db_aggregate_update_host, 2^21-element chunks, pinned host buffers",
+            "gpu_launches_per_step": nchunks + 1}
 
-    peak, peak_kind = measured_peak()
-    kernel_ms = float(np.mean(per_step_ms))
-    achieved = bytes_step / (kernel_ms * 1e-3) / 1e9
-    out = {
-        "metric": METRIC, "value": job_bps / 1e9, "unit": "GB/s",
-        "iterations_per_s": world * args.steps / (max_ms * 1e-3),
-        "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
-        "ms_per_step": max_ms / args.steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "K": K, "N": N, "grad_dtype": "f32", "global_batch": sum(B0),
-                   "kp": KP, "lr": LR, "mu": MU, "grad_sqnorm": True,
-                   "bytes_per_step": bytes_step, "l2": "inputs (1.23 GB per step) exceed the 126 MB L2",
-                   "parallelism": f"{world} independent replica(s), no collective"},
-        "e2e": {"value": e2e_bps / 1e9, "unit": "GB/s", "steps": e2e_steps,
-                "ms_per_step": e2e_ms / e2e_steps,
-                "h2d_bytes_per_step": K * N * 4, "d2h_bytes_per_step": N * 4 + 8},
-        "gpu_launches": args.steps,
-        "clocks": sampler.summary(),
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_source": f"of {peak_kind}",
-                     "kernel": "agg_vec_kernel<float, 8, 1, true>", "kernel_ms": kernel_ms,
-                     "kernel_ms_min": float(np.min(per_step_ms)), "traffic": kernel_traffic()},
-    }
-    if rank == 0 and world == 1:
-        del host_grads, host_p
-        out["cpu_baseline"] = cpu_baseline([g.cpu().numpy() for g in grads], b)
+
+def run_ours(args):
+    from paper_2305_12213_b200 import binding, build
+    rank, local_rank, world = replicas.env_world()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; libdynbatch has no CPU fallback")
+    dev = torch.device("cuda", local_rank if world > 1 else 0)
+    torch.cuda.set_device(dev)
+    replicas.init(device=dev)
     if rank == 0:
-        print(json.dumps(out), flush=True)
+        build.build()
+    replicas.barrier(dev)
+    binding.lib()
+    if args.workload == "sweep":
+        for wl in sweep_workloads():
+            out = measure(wl, args, dev, rank, world, with_e2e=False, with_cpu=False)
+            if rank == 0:
+                print(json.dumps(out), flush=True)
+            torch.cuda.empty_cache()
+    else:
+        out = measure(WORKLOADS[args.workload](), args, dev, rank, world)
+        if rank == 0:
+            print(json.dumps(out), flush=True)
     replicas.shutdown()
 
 
-def cpu_baseline(host_grads, b, budget_s: float = 15.0):
+def host_gradients(grads):
+    """Device gradient tensors -> the numpy arrays the oracle takes (fp32, or uint16 bf16 bit patterns)."""
+    out = []
+    for g in grads:
+        t = g.detach().cpu().contiguous()
+        out.append(t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy())
+    return out
+
+
+def cpu_baseline(wl, host_grads, b, budget_s: float = 15.0):
     """The fp64 oracle, as it stands, on the host cores, over the same workload (all N, all K)."""
     import oracle
-    N = host_grads[0].size
+    N = wl.N
     p = inputs.normal(N, PARAM_STD, 1, "cpu").numpy().astype(np.float64)
     v = np.zeros(N, dtype=np.float64)
-    oracle.aggregate_update(host_grads, b, p, v, LR, MU)          # warm-up pass
+    oracle.aggregate_update(host_grads, b, p, v, wl.lr, wl.mu)          # warm-up pass
     t0 = time.perf_counter()
     passes = 0
     while passes < 3 or (time.perf_counter() - t0 < budget_s and passes < 50):
-        oracle.aggregate_update(host_grads, b, p, v, LR, MU)
+        oracle.aggregate_update(host_grads, b, p, v, wl.lr, wl.mu)
         passes += 1
     dt = time.perf_counter() - t0
-    bytes_step = step_bytes(len(host_grads), N, 4)
-    return {"value": bytes_step * passes / dt / 1e9, "unit": "GB/s", "cores": oracle.num_threads(),
+    return {"value": wl.bytes_per_step * passes / dt / 1e9, "unit": "GB/s", "cores": oracle.num_threads(),
             "kind": "oracle", "iterations_per_s": passes / dt,
-            "sample": f"{passes} full passes of the workload (N={N}, K={len(host_grads)}), "
+            "sample": f"{passes} full passes of the workload (N={N}, K={wl.K}), "
                       "fp64 state, OpenMP over elements"}
 
 
@@ -270,25 +374,26 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle
-    K, N = K_WORKERS, N_PARAMS
+    wl = WORKLOADS[args.workload if args.workload != "sweep" else "resnet50"]()
+    K, N = wl.K, wl.N
     steps, warm = args.steps, max(1, args.warmup)
     probe_n = 1 << 20
-    host = [g.numpy() for g in inputs.worker_gradients(K, probe_n, GRAD_STD, 2000)]
+    host = host_gradients(inputs.worker_gradients(K, probe_n, wl.grad_std, 2000, dtype=wl.grad_dtype))
     pp, vv = np.zeros(probe_n), np.zeros(probe_n)
-    oracle.aggregate_update(host, B0, pp, vv, LR, MU)
+    oracle.aggregate_update(host, wl.b0, pp, vv, wl.lr, wl.mu)
     t0 = time.perf_counter()
-    oracle.aggregate_update(host, B0, pp, vv, LR, MU)
+    oracle.aggregate_update(host, wl.b0, pp, vv, wl.lr, wl.mu)
     per_elem = (time.perf_counter() - t0) / probe_n
     n = int(min(N, max(1 << 16, 90.0 / (steps + warm) / per_elem)))
-    host = [g.numpy() for g in inputs.worker_gradients(K, n, GRAD_STD, 2000)]
+    host = host_gradients(inputs.worker_gradients(K, n, wl.grad_std, 2000, dtype=wl.grad_dtype))
     p = inputs.normal(n, PARAM_STD, 2500).numpy().astype(np.float64)
     v = np.zeros(n)
-    b = np.array(B0, dtype=np.int32)
+    b = np.array(wl.b0, dtype=np.int32)
 
     def step():
         nonlocal b
-        b = oracle.controller_step(b, THROUGHPUTS, KP)
-        oracle.aggregate_update(host, b, p, v, LR, MU)
+        b = oracle.controller_step(b, wl.throughputs, wl.kp)
+        oracle.aggregate_update(host, b, p, v, wl.lr, wl.mu)
 
     for _ in range(warm):
         step()
@@ -296,8 +401,7 @@ def run_reference(args):
     for _ in range(steps):
         step()
     dt = time.perf_counter() - t0
-    bytes_step = step_bytes(K, n, 4)
-    val = bytes_step * steps / dt / 1e9
+    val = step_bytes(K, n, wl.grad_bytes) * steps / dt / 1e9
     sample = f"first {n} of {N} parameters per step, all K={K} workers, fp64 state"
     out = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s",
@@ -305,8 +409,9 @@ def run_reference(args):
         "n_gpus": args.gpus, "steps": steps, "warmup": warm, "ms_per_step": dt / steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
-        "config": {"workload": WORKLOAD, "K": K, "N": N, "grad_dtype": "f32", "global_batch": sum(B0),
-                   "kp": KP, "lr": LR, "mu": MU, "sample": sample},
+        "config": {"workload": wl.name, "K": K, "N": N,
+                   "grad_dtype": "f32" if wl.grad_dtype == torch.float32 else "bf16",
+                   "global_batch": sum(wl.b0), "kp": wl.kp, "lr": wl.lr, "mu": wl.mu, "sample": sample},
         "cpu_baseline": {"value": val, "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -321,6 +426,8 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=["resnet50", "bert_base", "small", "sweep"], default="resnet50",
+                    help="resnet50 is the headline configuration; sweep prints one line per (N, K) point")
     args = ap.parse_args()
     if args.steps < 1:
         raise SystemExit("--steps must be >= 1")

@@ -143,6 +143,56 @@ db_status db_aggregate_update_static(const void* const* grads,
                                      double* grad_sqnorm, void* cuda_stream);
 
 /* ------------------------------------------------------------------------
+ * The same step with the gradients in HOST memory   (Section 3.1, Eq. 2-3;
+ * in the paper's system the parameter server receives the workers' gradients
+ * over the network, i.e. in host buffers, and sends the new model back)
+ *
+ * db_aggregate_update_host cuts the N parameters into chunks and overlaps,
+ * chunk by chunk, the host->device copy of the K gradient slices, the fused
+ * aggregate/update kernel and the device->host copy of the updated
+ * parameters on three streams.  params/momentum stay resident on the device
+ * and are updated in place exactly as by db_aggregate_update_ex (bit-identical:
+ * the update is element-wise); the squared norm is the sum of the per-chunk
+ * norms in chunk order (same value to rounding).
+ *
+ *   pipeline         from db_host_pipeline_create on the current device; holds
+ *                    two side streams and events, no device memory.  One call at
+ *                    a time per pipeline.
+ *   host_grads       host array of K HOST pointers, N elements each; page-locked
+ *                    memory is needed for the copies to overlap (pageable memory
+ *                    works, serialised by the runtime).  b[k] == 0: never read.
+ *   params, momentum device, N fp32, in/out
+ *   host_params_out  host, N fp32, receives the updated parameters, or NULL
+ *   host_sqnorm_out  host, one double, or NULL
+ *   staging          device scratch of >= db_host_staging_bytes(K, dtype, N,
+ *                    chunk_elems) bytes, 256-byte aligned, uninitialised
+ *   chunk_elems      elements per chunk (rounded up to a multiple of 8);
+ *                    <= 0 selects the default of 2^21
+ *   cuda_stream      the kernels run here; the call is ordered after earlier work
+ *                    on it, and work enqueued on it afterwards starts only when
+ *                    every copy of this call has finished.  Host outputs are valid
+ *                    after synchronising this stream; host_grads must stay
+ *                    unchanged until then.
+ * ------------------------------------------------------------------------ */
+typedef struct db_host_pipeline db_host_pipeline;
+
+db_status db_host_pipeline_create(db_host_pipeline** out);
+db_status db_host_pipeline_destroy(db_host_pipeline* pipeline);
+
+size_t db_host_staging_bytes(int32_t K, db_dtype grad_dtype, int64_t N,
+                             int64_t chunk_elems);
+
+db_status db_aggregate_update_host(db_host_pipeline* pipeline,
+                                   const void* const* host_grads,
+                                   db_dtype grad_dtype, const int32_t* b,
+                                   int32_t K, int64_t N, float* params,
+                                   float* momentum, float lr, float mu,
+                                   float* host_params_out,
+                                   double* host_sqnorm_out, void* staging,
+                                   size_t staging_bytes, int64_t chunk_elems,
+                                   void* cuda_stream);
+
+/* ------------------------------------------------------------------------
  * Ragged per-worker gradient of a linear-softmax classifier
  *
  * The model on which the batch-proportional weighting of Eq. 2 is checked

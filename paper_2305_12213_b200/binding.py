@@ -41,6 +41,12 @@ _SIGNATURES = {
     "db_aggregate_workspace_bytes": (c_size_t, [c_int32, c_int64]),
     "db_aggregate_update_static": (c_int32, [c_void_p, c_int32, c_void_p, c_int32, c_int64, c_void_p,
                                              c_void_p, c_float, c_float, c_void_p, c_void_p]),
+    "db_host_pipeline_create": (c_int32, [c_void_p]),
+    "db_host_pipeline_destroy": (c_int32, [c_void_p]),
+    "db_host_staging_bytes": (c_size_t, [c_int32, c_int32, c_int64, c_int64]),
+    "db_aggregate_update_host": (c_int32, [c_void_p, c_void_p, c_int32, c_void_p, c_int32, c_int64, c_void_p,
+                                           c_void_p, c_float, c_float, c_void_p, c_void_p, c_void_p, c_size_t,
+                                           c_int64, c_void_p]),
     "db_worker_grad": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p,
                                  c_void_p, c_void_p, c_size_t, c_void_p]),
     "db_worker_grad_workspace_bytes": (c_size_t, [c_int32, c_int32, c_int32]),
@@ -152,6 +158,64 @@ def aggregate_update_static(grads: Sequence[torch.Tensor], b: Sequence[int], par
         ctypes.cast(_i32_array(b), c_void_p), K, int(params.numel()),
         _dev_ptr(params, torch.float32, "params"), _dev_ptr(momentum, torch.float32, "momentum"),
         float(lr), float(mu), _dev_ptr(grad_sqnorm, torch.float64, "grad_sqnorm"), _stream_ptr(stream)))
+
+
+def _dtype_code(dt: torch.dtype) -> int:
+    if dt == torch.float32:
+        return DB_F32
+    if dt == torch.bfloat16:
+        return DB_BF16
+    raise TypeError("gradients must be float32 or bfloat16")
+
+
+def host_staging_bytes(K: int, grad_dtype: torch.dtype, N: int, chunk_elems: int = 0) -> int:
+    return int(lib().db_host_staging_bytes(int(K), _dtype_code(grad_dtype), int(N), int(chunk_elems)))
+
+
+class HostPipeline:
+    """db_host_pipeline: side streams and events for db_aggregate_update_host on the current device."""
+
+    def __init__(self):
+        self._h = c_void_p()
+        _check(lib().db_host_pipeline_create(ctypes.byref(self._h)))
+
+    def close(self) -> None:
+        if self._h:
+            lib().db_host_pipeline_destroy(self._h)
+            self._h = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def aggregate_update(self, host_grads: Sequence[torch.Tensor], b: Sequence[int], params: torch.Tensor,
+                         momentum: torch.Tensor, lr: float, mu: float,
+                         host_params_out: Optional[torch.Tensor], host_sqnorm_out: Optional[torch.Tensor],
+                         staging: torch.Tensor, chunk_elems: int = 0,
+                         stream: Optional[torch.cuda.Stream] = None) -> None:
+        """db_aggregate_update_host: gradients in (pinned) host tensors, parameters copied back to the host."""
+        K = len(host_grads)
+        if len(b) != K:
+            raise ValueError("len(b) != len(host_grads)")
+        gdt = host_grads[0].dtype
+        for g in host_grads:
+            if g.is_cuda or g.dtype != gdt or not g.is_contiguous():
+                raise TypeError("host_grads must be contiguous CPU tensors of one dtype")
+        for t, dt, name in ((host_params_out, torch.float32, "host_params_out"),
+                            (host_sqnorm_out, torch.float64, "host_sqnorm_out")):
+            if t is not None and (t.is_cuda or t.dtype != dt or not t.is_contiguous()):
+                raise TypeError(f"{name} must be a contiguous CPU tensor of {dt}")
+        table = (c_void_p * K)(*[g.data_ptr() for g in host_grads])
+        _check(lib().db_aggregate_update_host(
+            self._h, ctypes.cast(table, c_void_p), _dtype_code(gdt), ctypes.cast(_i32_array(b), c_void_p), K,
+            int(params.numel()), _dev_ptr(params, torch.float32, "params"),
+            _dev_ptr(momentum, torch.float32, "momentum"), float(lr), float(mu),
+            None if host_params_out is None else host_params_out.data_ptr(),
+            None if host_sqnorm_out is None else host_sqnorm_out.data_ptr(),
+            staging.data_ptr(), staging.numel() * staging.element_size(), int(chunk_elems),
+            _stream_ptr(stream)))
 
 
 def worker_grad_workspace_bytes(b_i: int, D: int, C: int) -> int:
