@@ -210,16 +210,58 @@ db_status db_aggregate_update_host(db_host_pipeline* pipeline,
  *   G     device [D, C] row-major fp32, overwritten
  *   loss  device, one float (mean cross-entropy), or NULL
  *   workspace  device scratch of >= db_worker_grad_workspace_bytes(b_i, D, C)
- *         bytes, 16-byte aligned, uninitialised
- * X, W, G must be 16-byte aligned when D and C are multiples of 4 (they are
- * for any whole allocation); other shapes take element-wise loads.
+ *         bytes, 16-byte aligned, uninitialised.  Its first 32-bit word is a
+ *         status word the call clears and the tensor-core kernels set to a
+ *         non-zero code if one of their (time-limited) internal waits ever
+ *         gives up; it stays 0 in correct operation.
+ *   flags 0, or DB_WORKER_GRAD_FFMA to run both contractions as plain fp32
+ *         FFMA instead of on the tensor cores (the accuracy reference; also
+ *         taken automatically for b_i > 4096)
+ * Any D, C and alignment down to 4 bytes are accepted; 16-byte aligned X with
+ * D a multiple of 4 takes 128-bit loads.
+ *
+ * On the tensor cores every fp32 product is formed from three TF32 products
+ * (operands split into two TF32 halves, fp32 accumulation), which keeps the
+ * result within 1e-5 of an fp64 evaluation.
+ * db_worker_grad is db_worker_grad_ex with flags = 0.
  * ------------------------------------------------------------------------ */
+#define DB_WORKER_GRAD_FFMA 1u
+
 db_status db_worker_grad(const float* X, const int32_t* y, const float* W,
                          int32_t b_i, int32_t D, int32_t C, float* G,
                          float* loss, void* workspace, size_t workspace_bytes,
                          void* cuda_stream);
 
+db_status db_worker_grad_ex(const float* X, const int32_t* y, const float* W,
+                            int32_t b_i, int32_t D, int32_t C, float* G,
+                            float* loss, void* workspace,
+                            size_t workspace_bytes, uint32_t flags,
+                            void* cuda_stream);
+
 size_t db_worker_grad_workspace_bytes(int32_t b_i, int32_t D, int32_t C);
+
+/* ------------------------------------------------------------------------
+ * The dense fp32 contraction db_worker_grad is built from (both Z = X W and
+ * G = X^T E are instances), exposed so that it can be checked in isolation:
+ *     out(m, n) = sum_{k < K} A(m, k) * B(n, k)
+ * on the tensor cores with three TF32 products per fp32 product.
+ *
+ *   A(m, k) = A[m * a_row + k * a_k],  B(n, k) = B[n * b_row + k * b_k]
+ *   out(m, n) at out[m * o_m + n * o_n]       all device fp32, strides in
+ *   elements, >= 0 (outputs >= 1); either operand may be contiguous along k or
+ *   along its rows, which selects 128-bit loads when 16-byte aligned.
+ *   M, N >= 1, K >= 0 (K = 0 writes zeros)
+ *   status   device, one int32 the caller has cleared; set non-zero if a
+ *            time-limited wait inside the kernel gave up
+ * The tensor core truncates when it adds into its fp32 accumulator (measured
+ * bias 7e-9 * chain length, relative), so the reduction is dealt round-robin to
+ * up to 15 accumulators in tensor memory that are added at the end in fp32.
+ * ------------------------------------------------------------------------ */
+db_status db_contract_f32(const float* A, int64_t a_row, int64_t a_k,
+                          const float* B, int64_t b_row, int64_t b_k,
+                          float* out, int64_t o_m, int64_t o_n, int32_t M,
+                          int32_t N, int32_t K, int32_t* status,
+                          void* cuda_stream);
 
 /* ------------------------------------------------------------------------
  * Proportional batch-size controller, host side   (Section 3.3, Eq. 4-5)

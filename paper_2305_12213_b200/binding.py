@@ -49,6 +49,10 @@ _SIGNATURES = {
                                            c_int64, c_void_p]),
     "db_worker_grad": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p,
                                  c_void_p, c_void_p, c_size_t, c_void_p]),
+    "db_worker_grad_ex": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p,
+                                    c_void_p, c_void_p, c_size_t, ctypes.c_uint32, c_void_p]),
+    "db_contract_f32": (c_int32, [c_void_p, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p, c_int64,
+                                  c_int64, c_int32, c_int32, c_int32, c_void_p, c_void_p]),
     "db_worker_grad_workspace_bytes": (c_size_t, [c_int32, c_int32, c_int32]),
     "db_controller_step": (c_int32, [c_void_p, c_void_p, c_int32, c_double]),
     "db_controller_step_ex": (c_int32, [c_void_p, c_void_p, c_int32, c_double, c_void_p, c_void_p]),
@@ -222,20 +226,43 @@ def worker_grad_workspace_bytes(b_i: int, D: int, C: int) -> int:
     return int(lib().db_worker_grad_workspace_bytes(int(b_i), int(D), int(C)))
 
 
+DB_WORKER_GRAD_FFMA = 1
+
+
 def worker_grad(X: torch.Tensor, y: torch.Tensor, W: torch.Tensor, G: torch.Tensor,
                 loss: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
-                stream: Optional[torch.cuda.Stream] = None) -> None:
-    """db_worker_grad: G = X^T (softmax(X W) - onehot(y)) / b_i, optional mean cross-entropy."""
+                stream: Optional[torch.cuda.Stream] = None, flags: int = 0) -> None:
+    """db_worker_grad_ex: G = X^T (softmax(X W) - onehot(y)) / b_i, optional mean cross-entropy."""
     b_i, D = X.shape
     D2, C = W.shape
     if D2 != D or tuple(G.shape) != (D, C) or y.numel() != b_i:
         raise ValueError("shape mismatch")
-    _check(lib().db_worker_grad(
+    _check(lib().db_worker_grad_ex(
         _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.int32, "y"), _dev_ptr(W, torch.float32, "W"),
         b_i, D, C, _dev_ptr(G, torch.float32, "G"), _dev_ptr(loss, torch.float32, "loss"),
         None if workspace is None else workspace.data_ptr(),
         0 if workspace is None else workspace.numel() * workspace.element_size(),
-        _stream_ptr(stream)))
+        int(flags), _stream_ptr(stream)))
+
+
+def contract_f32(A: torch.Tensor, B: torch.Tensor, out: torch.Tensor, status: torch.Tensor,
+                 stream: Optional[torch.cuda.Stream] = None) -> None:
+    """db_contract_f32: out[m, n] = sum_k A[m, k] * B[n, k] for 2-D fp32 CUDA tensors of any strides."""
+    M, K = A.shape
+    N, K2 = B.shape
+    if K2 != K or tuple(out.shape) != (M, N):
+        raise ValueError("shape mismatch")
+    for t in (A, B, out):
+        if not t.is_cuda or t.dtype != torch.float32:
+            raise TypeError("A, B, out must be float32 CUDA tensors")
+    _check(lib().db_contract_f32(
+        A.data_ptr(), A.stride(0), A.stride(1), B.data_ptr(), B.stride(0), B.stride(1), out.data_ptr(),
+        out.stride(0), out.stride(1), M, N, K, _dev_ptr(status, torch.int32, "status"), _stream_ptr(stream)))
+
+
+def worker_grad_status(workspace: torch.Tensor) -> int:
+    """The status word at the start of a db_worker_grad workspace (0 = every internal wait completed)."""
+    return int(workspace[:4].view(torch.int32).item())
 
 
 def controller_step(b: Sequence[int], throughputs: Sequence[float], kp: float,

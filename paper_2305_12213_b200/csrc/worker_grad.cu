@@ -8,12 +8,14 @@
 //      handful of rows still fills the GPU; partial sums go to the workspace;
 //   2. softmax: one CTA per sample folds the partials in split order, applies
 //      the max-subtracted softmax, subtracts the one-hot label, scales by 1/b_i;
-//   3. gradient: G = X^T E, one 64x64 output tile per CTA, reduction depth b_i.
-// Both contractions are fp32 FFMA on shared-memory tiles: at b_i <= 128 they
-// sit below the tensor-core ridge (bounded by reading W and writing G).
+//   3. gradient: G = X^T E, reduction depth b_i.
+// The two contractions run on the tensor cores (tcgen05, three TF32 products per
+// fp32 product, see tc_gemm.cuh).  An fp32 FFMA version on shared-memory tiles is
+// kept as the accuracy reference and for very large b_i.
 #include <cstdint>
 
 #include "common.h"
+#include "tc_gemm.cuh"
 
 namespace dynbatch {
 namespace {
@@ -149,44 +151,107 @@ __device__ __forceinline__ float block_reduce(float x, float* smem, bool take_ma
     return r;  // same value in every thread
 }
 
-// One CTA per sample i:  E[i, :] = (softmax(z_i) - onehot(y_i)) / b,  z_i = sum of the split partials.
+// One CTA per sample i:  E[i, :] = (softmax(z_i) - onehot(y_i)) / b,  z_i = sum of the split partials
+// (split order).  The last CTA to finish also folds the per-sample losses into the mean loss; arrival
+// order comes from an atomic ticket (zeroed by the caller), nobody waits.
+// IN_REGS: C <= 4 * kThreads, every thread keeps its four logits in registers (one pass over memory);
+// otherwise the logits are parked in E between the passes.
+template <bool IN_REGS>
 __global__ void __launch_bounds__(kThreads)
 softmax_residual_kernel(const float* __restrict__ partials, int splits, long long split_stride,
                         const int32_t* __restrict__ y, float* __restrict__ E, float* __restrict__ row_loss,
-                        int b, int C) {
+                        int b, int C, unsigned int* __restrict__ ticket, float* __restrict__ loss) {
     __shared__ float smem[kThreads / 32];
+    __shared__ float z_label;
+    __shared__ bool is_last;
     const int i = blockIdx.x;
     float* e = E + static_cast<long long>(i) * C;
     const float* z0 = partials + static_cast<long long>(i) * C;
+    const int label = y[i];
+    const float inv_b = 1.0f / static_cast<float>(b);
     float zmax = -INFINITY;
-    for (int c = threadIdx.x; c < C; c += kThreads) {
-        float z = 0.0f;
-        for (int s = 0; s < splits; ++s) z += z0[static_cast<long long>(s) * split_stride + c];
-        e[c] = z;
-        zmax = fmaxf(zmax, z);
+    float z[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    if (threadIdx.x == 0) z_label = 0.0f;
+    // four classes per thread and eight splits per round: 32 independent loads in flight, adds in split order
+    for (int cb = 0; cb < C; cb += 4 * kThreads) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) z[j] = 0.0f;
+        for (int s0 = 0; s0 < splits; s0 += 8) {
+            float t[4][8];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int c = cb + j * kThreads + threadIdx.x;
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    t[j][u] = (c < C && s0 + u < splits)
+                                  ? __ldg(z0 + static_cast<long long>(s0 + u) * split_stride + c) : 0.0f;
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (s0 + u < splits) z[j] += t[j][u];
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = cb + j * kThreads + threadIdx.x;
+            if (c < C) {
+                if (!IN_REGS) e[c] = z[j];
+                zmax = fmaxf(zmax, z[j]);
+            }
+        }
     }
     zmax = block_reduce(zmax, smem, true);
     float den = 0.0f;
-    for (int c = threadIdx.x; c < C; c += kThreads) den += expf(e[c] - zmax);
-    den = block_reduce(den, smem, false);
-    const int label = y[i];
-    const float inv_b = 1.0f / static_cast<float>(b);
+    if (IN_REGS) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = j * kThreads + threadIdx.x;
+            if (c < C) {
+                z[j] = expf(z[j] - zmax);       // numerator of the softmax
+                den += z[j];
+                if (c == label) z_label = z[j];
+            }
+        }
+    } else {
+        for (int c = threadIdx.x; c < C; c += kThreads) {
+            const float p = expf(e[c] - zmax);
+            den += p;
+            if (c == label) z_label = p;
+        }
+    }
+    den = block_reduce(den, smem, false);       // its barriers also publish z_label
     if (threadIdx.x == 0)
-        row_loss[i] = (label >= 0 && label < C) ? -((e[label] - zmax) - logf(den)) : 0.0f;
-    __syncthreads();  // e[label] read above before it is overwritten below
-    for (int c = threadIdx.x; c < C; c += kThreads) {
-        float r = expf(e[c] - zmax) / den;
-        if (c == label) r -= 1.0f;
-        e[c] = r * inv_b;
+        row_loss[i] = (label >= 0 && label < C) ? -logf(z_label / den) : 0.0f;
+    if (IN_REGS) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = j * kThreads + threadIdx.x;
+            if (c < C) {
+                float r = z[j] / den;
+                if (c == label) r -= 1.0f;
+                e[c] = r * inv_b;
+            }
+        }
+    } else {
+        for (int c = threadIdx.x; c < C; c += kThreads) {
+            float r = expf(e[c] - zmax) / den;
+            if (c == label) r -= 1.0f;
+            e[c] = r * inv_b;
+        }
     }
-}
-
-__global__ void mean_loss_kernel(const float* __restrict__ row_loss, int b, float* __restrict__ loss) {
-    if (threadIdx.x == 0 && blockIdx.x == 0) {
-        float s = 0.0f;
-        for (int i = 0; i < b; ++i) s += row_loss[i];
-        *loss = s / static_cast<float>(b);
+    if (loss == nullptr) return;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        is_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
     }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    float part = 0.0f;
+    for (int r = threadIdx.x; r < b; r += kThreads) part += __ldcg(row_loss + r);
+    const float total = block_reduce(part, smem, false);
+    if (threadIdx.x == 0) *loss = total * inv_b;
 }
 
 size_t round16(size_t x) { return (x + 15) & ~static_cast<size_t>(15); }
@@ -202,18 +267,39 @@ int logit_splits(int b, int D, int C) {
     return static_cast<int>(s);
 }
 
+constexpr int kMaxTensorCoreBatch = 4096;  // longer reductions over the batch go to FFMA
+constexpr size_t kStatusBytes = 16;        // device status word of the tensor-core kernels
+
 struct WorkerLayout {
+    bool tensor;            // tensor-core path
     int splits, k_per_split;
+    int n_tile;             // accumulator columns of the logits GEMM (tensor path)
     size_t partial_bytes, e_bytes, loss_bytes;
+    size_t total() const { return kStatusBytes + partial_bytes + e_bytes + loss_bytes; }
 };
 
-WorkerLayout layout_for(int b, int D, int C) {
+WorkerLayout layout_for(int b, int D, int C, bool tensor) {
     WorkerLayout L;
-    L.splits = logit_splits(b, D, C);
-    int per = (D + L.splits - 1) / L.splits;
-    per = (per + kDepth - 1) / kDepth * kDepth;  // whole stages, keeps 16-byte alignment of k offsets
-    L.k_per_split = per;
-    L.splits = (D + per - 1) / per;
+    L.tensor = tensor;
+    L.n_tile = b <= 32 ? 32 : (b <= 64 ? 64 : 128);
+    if (tensor) {
+        // logits are computed transposed: 128 classes x n_tile samples per CTA, split over D so that
+        // about one CTA per SM exists; splits are whole 32-feature blocks
+        const long long tiles = static_cast<long long>((C + tc::kTileM - 1) / tc::kTileM) * ((b + L.n_tile - 1) / L.n_tile);
+        long long s = sm_count() / tiles;
+        const int kblocks = (D + tc::kBlockK - 1) / tc::kBlockK;
+        if (s > kblocks) s = kblocks;
+        if (s < 1) s = 1;
+        const int per_blocks = static_cast<int>((kblocks + s - 1) / s);
+        L.k_per_split = per_blocks * tc::kBlockK;
+        L.splits = (D + L.k_per_split - 1) / L.k_per_split;
+    } else {
+        L.splits = logit_splits(b, D, C);
+        int per = (D + L.splits - 1) / L.splits;
+        per = (per + kDepth - 1) / kDepth * kDepth;  // whole stages, keeps 16-byte alignment of k offsets
+        L.k_per_split = per;
+        L.splits = (D + per - 1) / per;
+    }
     L.partial_bytes = round16(sizeof(float) * static_cast<size_t>(L.splits) * b * C);
     L.e_bytes = round16(sizeof(float) * static_cast<size_t>(b) * C);
     L.loss_bytes = round16(sizeof(float) * static_cast<size_t>(b));
@@ -222,36 +308,122 @@ WorkerLayout layout_for(int b, int D, int C) {
 
 bool valid_shape(int b, int D, int C) { return b >= 1 && b <= 65535 && D >= 1 && C >= 1; }
 
+using TcKernel = void (*)(const tc::GemmArgs);
+
+template <int N_TILE, int MODE_A>
+TcKernel pick_tc_b(int mode_b) {
+    switch (mode_b) {
+        case tc::kLoadKVec: return tc::tf32x3_gemm_kernel<N_TILE, MODE_A, tc::kLoadKVec>;
+        case tc::kLoadRowVec: return tc::tf32x3_gemm_kernel<N_TILE, MODE_A, tc::kLoadRowVec>;
+        default: return tc::tf32x3_gemm_kernel<N_TILE, MODE_A, tc::kLoadScalar>;
+    }
+}
+
+template <int N_TILE>
+TcKernel pick_tc(int mode_a, int mode_b) {
+    switch (mode_a) {
+        case tc::kLoadKVec: return pick_tc_b<N_TILE, tc::kLoadKVec>(mode_b);
+        case tc::kLoadRowVec: return pick_tc_b<N_TILE, tc::kLoadRowVec>(mode_b);
+        default: return pick_tc_b<N_TILE, tc::kLoadScalar>(mode_b);
+    }
+}
+
+// Widest loader the operand's strides and alignment allow.
+int load_mode(const float* p, long long row_stride, long long k_stride) {
+    const bool base16 = reinterpret_cast<uintptr_t>(p) % 16 == 0;
+    if (k_stride == 1 && row_stride % 4 == 0 && base16) return tc::kLoadKVec;
+    if (row_stride == 1 && k_stride % 4 == 0 && base16) return tc::kLoadRowVec;
+    return tc::kLoadScalar;
+}
+
+// out(m, n) = sum_k A(m, k) B(n, k) on the tensor cores; a.k_per_split must be a multiple of 32.
+db_status launch_tc_gemm(tc::GemmArgs a, int n_tile, cudaStream_t stream) {
+    if (n_tile != 32 && n_tile != 64) n_tile = 128;
+    // one main accumulator per four reduction blocks (chains of 16 additions), within 512 columns
+    const int blocks = a.k_per_split / tc::kBlockK;
+    int n_acc = (blocks + 3) / 4;
+    if (n_acc > 512 / n_tile - 1) n_acc = 512 / n_tile - 1;
+    a.n_acc = n_acc < 1 ? 1 : n_acc;
+    const int mode_a = load_mode(a.A, a.a_row, a.a_k), mode_b = load_mode(a.B, a.b_row, a.b_k);
+    TcKernel fn;
+    int smem;
+    switch (n_tile) {
+        case 32: fn = pick_tc<32>(mode_a, mode_b); smem = tc::SmemLayout<32>::kBytes; break;
+        case 64: fn = pick_tc<64>(mode_a, mode_b); smem = tc::SmemLayout<64>::kBytes; break;
+        default: fn = pick_tc<128>(mode_a, mode_b); smem = tc::SmemLayout<128>::kBytes; n_tile = 128; break;
+    }
+    DB_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    const int splits = a.k_per_split > 0 ? (a.K + a.k_per_split - 1) / a.k_per_split : 1;
+    dim3 grid((a.N + n_tile - 1) / n_tile, (a.M + tc::kTileM - 1) / tc::kTileM, splits < 1 ? 1 : splits);
+    fn<<<grid, tc::kThreads, smem, stream>>>(a);
+    DB_CUDA_TRY(cudaGetLastError());
+    return DB_OK;
+}
+
+bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
+
 }  // namespace
 }  // namespace dynbatch
+
+extern "C" db_status db_contract_f32(const float* A, int64_t a_row, int64_t a_k, const float* B, int64_t b_row,
+                                     int64_t b_k, float* out, int64_t o_m, int64_t o_n, int32_t M, int32_t N,
+                                     int32_t K, int32_t* status, void* cuda_stream) {
+    using namespace dynbatch;
+    if (!A || !B || !out || !status) return DB_ERR_NULL;
+    if (M < 1 || N < 1 || K < 0) return DB_ERR_ARG;
+    if (a_row < 0 || a_k < 0 || b_row < 0 || b_k < 0 || o_m < 1 || o_n < 1) return DB_ERR_ARG;
+    if (reinterpret_cast<uintptr_t>(A) % 4 || reinterpret_cast<uintptr_t>(B) % 4 ||
+        reinterpret_cast<uintptr_t>(out) % 4 || reinterpret_cast<uintptr_t>(status) % 4)
+        return DB_ERR_ARG;
+    tc::GemmArgs a{};
+    a.A = A; a.a_row = a_row; a.a_k = a_k;
+    a.B = B; a.b_row = b_row; a.b_k = b_k;
+    a.out = out; a.o_m = o_m; a.o_n = o_n; a.o_split = 0;
+    a.M = M; a.N = N; a.K = K;
+    a.k_per_split = K > 0 ? (K + tc::kBlockK - 1) / tc::kBlockK * tc::kBlockK : tc::kBlockK;
+    a.status = status;
+    return launch_tc_gemm(a, N <= 32 ? 32 : (N <= 64 ? 64 : 128), static_cast<cudaStream_t>(cuda_stream));
+}
 
 extern "C" size_t db_worker_grad_workspace_bytes(int32_t b_i, int32_t D, int32_t C) {
     using namespace dynbatch;
     if (!valid_shape(b_i, D, C)) return 0;
-    const WorkerLayout L = layout_for(b_i, D, C);
-    return L.partial_bytes + L.e_bytes + L.loss_bytes;
+    const size_t a = layout_for(b_i, D, C, true).total(), f = layout_for(b_i, D, C, false).total();
+    return a > f ? a : f;
 }
 
-extern "C" db_status db_worker_grad(const float* X, const int32_t* y, const float* W, int32_t b_i,
-                                    int32_t D, int32_t C, float* G, float* loss, void* workspace,
-                                    size_t workspace_bytes, void* cuda_stream) {
+extern "C" db_status db_worker_grad_ex(const float* X, const int32_t* y, const float* W, int32_t b_i,
+                                       int32_t D, int32_t C, float* G, float* loss, void* workspace,
+                                       size_t workspace_bytes, uint32_t flags, void* cuda_stream) {
     using namespace dynbatch;
     if (!X || !y || !W || !G || !workspace) return DB_ERR_NULL;
     if (!valid_shape(b_i, D, C)) return DB_ERR_ARG;
+    if (flags & ~static_cast<uint32_t>(DB_WORKER_GRAD_FFMA)) return DB_ERR_ARG;
     if (reinterpret_cast<uintptr_t>(workspace) % 16) return DB_ERR_ARG;
-    const WorkerLayout L = layout_for(b_i, D, C);
-    if (workspace_bytes < L.partial_bytes + L.e_bytes + L.loss_bytes) return DB_ERR_ARG;
+    if (workspace_bytes < db_worker_grad_workspace_bytes(b_i, D, C)) return DB_ERR_ARG;
+    const bool tensor = !(flags & DB_WORKER_GRAD_FFMA) && b_i <= kMaxTensorCoreBatch;
+    const WorkerLayout L = layout_for(b_i, D, C, tensor);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
-    float* partials = static_cast<float*>(workspace);
-    float* E = reinterpret_cast<float*>(static_cast<char*>(workspace) + L.partial_bytes);
-    float* row_loss = reinterpret_cast<float*>(static_cast<char*>(workspace) + L.partial_bytes + L.e_bytes);
-    const bool vec4 = (D % 4 == 0) && (C % 4 == 0) && reinterpret_cast<uintptr_t>(X) % 16 == 0 &&
-                      reinterpret_cast<uintptr_t>(W) % 16 == 0 && reinterpret_cast<uintptr_t>(G) % 16 == 0;
+    char* base = static_cast<char*>(workspace);
+    int* status = reinterpret_cast<int*>(base);
+    float* partials = reinterpret_cast<float*>(base + kStatusBytes);
+    float* E = reinterpret_cast<float*>(base + kStatusBytes + L.partial_bytes);
+    float* row_loss = reinterpret_cast<float*>(base + kStatusBytes + L.partial_bytes + L.e_bytes);
     const long long bc = static_cast<long long>(b_i) * C;
+    DB_CUDA_TRY(cudaMemsetAsync(status, 0, kStatusBytes, stream));
 
     // 1. logits, split over D
-    {
+    if (tensor) {
+        tc::GemmArgs a{};
+        a.A = W; a.a_row = 1; a.a_k = C;          // A(m = class, k = feature) = W[k, m]
+        a.B = X; a.b_row = D; a.b_k = 1;          // B(n = sample, k = feature) = X[n, k]
+        a.out = partials; a.o_m = 1; a.o_n = C; a.o_split = bc;   // Z[n, m], one slab per split
+        a.M = C; a.N = b_i; a.K = D; a.k_per_split = L.k_per_split; a.status = status;
+        const db_status st = launch_tc_gemm(a, L.n_tile, stream);
+        if (st != DB_OK) return st;
+    } else {
+        const bool vec4 = (D % 4 == 0) && (C % 4 == 0) && aligned16(X) && aligned16(W);
         dim3 grid((C + kTile - 1) / kTile, (b_i + kTile - 1) / kTile, L.splits);
         if (vec4)
             tile_gemm_kernel<false, true><<<grid, kThreads, 0, stream>>>(X, D, W, C, partials, C, bc, b_i, C, D,
@@ -262,10 +434,26 @@ extern "C" db_status db_worker_grad(const float* X, const int32_t* y, const floa
         DB_CUDA_TRY(cudaGetLastError());
     }
     // 2. softmax residual (P - Y) / b
-    softmax_residual_kernel<<<b_i, kThreads, 0, stream>>>(partials, L.splits, bc, y, E, row_loss, b_i, C);
+    if (C <= 4 * kThreads)
+        softmax_residual_kernel<true><<<b_i, kThreads, 0, stream>>>(partials, L.splits, bc, y, E, row_loss, b_i, C,
+                                                                    reinterpret_cast<unsigned int*>(status) + 1, loss);
+    else
+        softmax_residual_kernel<false><<<b_i, kThreads, 0, stream>>>(partials, L.splits, bc, y, E, row_loss, b_i, C,
+                                                                     reinterpret_cast<unsigned int*>(status) + 1, loss);
     DB_CUDA_TRY(cudaGetLastError());
     // 3. G = X^T E
-    {
+    if (tensor) {
+        tc::GemmArgs a{};
+        a.A = X; a.a_row = 1; a.a_k = D;          // A(m = feature, k = sample) = X[k, m]
+        a.B = E; a.b_row = 1; a.b_k = C;          // B(n = class, k = sample) = E[k, n]
+        a.out = G; a.o_m = C; a.o_n = 1; a.o_split = 0;
+        a.M = D; a.N = C; a.K = b_i;
+        a.k_per_split = (b_i + tc::kBlockK - 1) / tc::kBlockK * tc::kBlockK;   // one split
+        a.status = status;
+        const db_status st = launch_tc_gemm(a, 64, stream);
+        if (st != DB_OK) return st;
+    } else {
+        const bool vec4 = (D % 4 == 0) && (C % 4 == 0) && aligned16(X) && aligned16(G);
         dim3 grid((C + kTile - 1) / kTile, (D + kTile - 1) / kTile, 1);
         if (vec4)
             tile_gemm_kernel<true, true><<<grid, kThreads, 0, stream>>>(X, D, E, C, G, C, 0, D, C, b_i, b_i);
@@ -273,9 +461,11 @@ extern "C" db_status db_worker_grad(const float* X, const int32_t* y, const floa
             tile_gemm_kernel<true, false><<<grid, kThreads, 0, stream>>>(X, D, E, C, G, C, 0, D, C, b_i, b_i);
         DB_CUDA_TRY(cudaGetLastError());
     }
-    if (loss) {
-        mean_loss_kernel<<<1, 32, 0, stream>>>(row_loss, b_i, loss);
-        DB_CUDA_TRY(cudaGetLastError());
-    }
     return DB_OK;
+}
+
+extern "C" db_status db_worker_grad(const float* X, const int32_t* y, const float* W, int32_t b_i,
+                                    int32_t D, int32_t C, float* G, float* loss, void* workspace,
+                                    size_t workspace_bytes, void* cuda_stream) {
+    return db_worker_grad_ex(X, y, W, b_i, D, C, G, loss, workspace, workspace_bytes, 0, cuda_stream);
 }

@@ -12,22 +12,28 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-def _worker_grad(X, y, W):
+TENSOR, FFMA = 0, binding.DB_WORKER_GRAD_FFMA
+
+
+def _worker_grad(X, y, W, flags=TENSOR):
     b_i, D = X.shape
     C = W.shape[1]
-    G = torch.empty(D, C, device=DEV)
+    G = torch.full((D, C), float("nan"), device=DEV)
     loss = torch.zeros(1, device=DEV)
     ws = torch.empty(binding.worker_grad_workspace_bytes(b_i, D, C), dtype=torch.uint8, device=DEV)
-    binding.worker_grad(X, y, W, G, loss, ws)
+    binding.worker_grad(X, y, W, G, loss, ws, flags=flags)
     torch.cuda.synchronize()
+    assert binding.worker_grad_status(ws) == 0, "a bounded wait inside the tensor-core kernel gave up"
     return G, float(loss.item())
 
 
+@pytest.mark.parametrize("flags", [TENSOR, FFMA])
 @pytest.mark.parametrize("b_i,D,C", [(1, 4, 4), (5, 6, 3), (7, 33, 10), (24, 128, 64), (3, 257, 130),
-                                      (65, 200, 96), (130, 64, 1000), (40, 2048, 1000)])
-def test_shapes_including_ragged_tiles(b_i, D, C):
+                                      (65, 200, 96), (130, 64, 1000), (40, 2048, 1000), (33, 100, 129),
+                                      (300, 96, 40), (128, 2048, 1000)])
+def test_shapes_including_ragged_tiles(b_i, D, C, flags):
     X, y, W = inputs.softmax_problem([b_i], D, C, seed=100 + b_i, w_std=0.05, device=DEV)
-    G, loss = _worker_grad(X, y, W)
+    G, loss = _worker_grad(X, y, W, flags)
     rG, rloss = oracle.worker_grad(X.cpu().numpy(), y.cpu().numpy(), W.cpu().numpy())
     assert rel_err(f64(G), rG) <= FP32_TOL
     assert abs(loss - rloss) <= FP32_TOL * abs(rloss)
@@ -38,13 +44,34 @@ def test_out_of_range_label_contributes_no_onehot():
     X, y, W = inputs.softmax_problem([4], 16, 8, seed=7, w_std=0.1, device=DEV)
     y2 = y.clone()
     y2[1] = 99
-    G, _ = _worker_grad(X, y2, W)
+    G, _ = _worker_grad(X, y2, W, FFMA)
     # the row sums of P alone are 1: column-sum identity is broken exactly by sample 1's features
     excess = G.double().sum(dim=1) * 4
     assert rel_err(excess.cpu().numpy(), f64(X[1])) <= 1e-5
 
 
-def test_config_ragged_four_workers_against_the_concatenated_batch():
+def test_misaligned_inputs_take_the_element_wise_loaders():
+    b_i, D, C = 19, 70, 37                      # D, C not multiples of 4; X shifted off 16-byte alignment
+    X, y, W = inputs.softmax_problem([b_i], D, C, seed=77, w_std=0.1, device=DEV)
+    Xs = torch.empty(b_i * D + 1, device=DEV)[1:].view(b_i, D)
+    Xs.copy_(X)
+    for flags in (TENSOR, FFMA):
+        G, loss = _worker_grad(Xs, y, W, flags)
+        rG, rloss = oracle.worker_grad(X.cpu().numpy(), y.cpu().numpy(), W.cpu().numpy())
+        assert rel_err(f64(G), rG) <= FP32_TOL and abs(loss - rloss) <= FP32_TOL * abs(rloss)
+
+
+def test_tensor_and_ffma_paths_agree_and_repeat_bitwise():
+    X, y, W = inputs.softmax_problem([64], 512, 250, seed=78, device=DEV)
+    G1, _ = _worker_grad(X, y, W, TENSOR)
+    G2, _ = _worker_grad(X, y, W, TENSOR)
+    G3, _ = _worker_grad(X, y, W, FFMA)
+    assert torch.equal(G1, G2)
+    assert rel_err(f64(G1), f64(G3)) <= FP32_TOL
+
+
+@pytest.mark.parametrize("flags", [TENSOR, FFMA])
+def test_config_ragged_four_workers_against_the_concatenated_batch(flags):
     """D=2048, C=1000, b={24,40,64,128}: per-worker gradients, then the weighted aggregate,
     which must be the mean gradient of all 256 samples."""
     bs = [24, 40, 64, 128]
@@ -55,7 +82,7 @@ def test_config_ragged_four_workers_against_the_concatenated_batch():
     Gs = []
     for i, b_i in enumerate(bs):
         s, e = int(offs[i]), int(offs[i + 1])
-        G, loss = _worker_grad(X[s:e].contiguous(), y[s:e].contiguous(), W)
+        G, loss = _worker_grad(X[s:e].contiguous(), y[s:e].contiguous(), W, flags)
         rG, rloss = oracle.worker_grad(Xh[s:e], yh[s:e], Wh)
         assert rel_err(f64(G), rG) <= FP32_TOL, f"worker {i}"
         assert abs(loss - rloss) <= FP32_TOL * abs(rloss)
