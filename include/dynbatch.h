@@ -241,6 +241,40 @@ db_status db_worker_grad_ex(const float* X, const int32_t* y, const float* W,
 size_t db_worker_grad_workspace_bytes(int32_t b_i, int32_t D, int32_t C);
 
 /* ------------------------------------------------------------------------
+ * All K workers' ragged gradients in three launches
+ *
+ * The workers of one iteration share W, so their logits are one contraction
+ * over the concatenated mini-batches; only the 1/b_w scale and the final
+ * reduction over each worker's own rows differ.  Worker w owns rows
+ * [offsets[w], offsets[w+1]) of X and y (its b_w = their number, Eq. 2's b_k)
+ * and receives G[w] = X_w^T (softmax(X_w W) - Y_w) / b_w and losses[w].
+ *
+ *   X        device [offsets[K], D] row-major fp32, the workers' rows in order
+ *   y        device [offsets[K]] int32
+ *   W        device [D, C] row-major fp32
+ *   offsets  host, K + 1 entries, offsets[0] = 0, strictly increasing (every
+ *            worker has at least one sample; at most 4096 per worker:
+ *            DB_ERR_UNSUPPORTED beyond)
+ *   K        1..DB_MAX_K
+ *   G        host array of K device pointers, each [D, C] fp32, overwritten
+ *   losses   device, K floats (mean cross-entropy per worker), or NULL
+ *   workspace  device scratch of >= db_worker_grad_grouped_workspace_bytes(
+ *            offsets[K], K, D, C) bytes, 16-byte aligned, uninitialised; its
+ *            first word is the status word described for db_worker_grad_ex
+ * Tensor-core path only; results equal db_worker_grad's on each worker to
+ * within the fp32 rounding of a differently split reduction over D.
+ * ------------------------------------------------------------------------ */
+db_status db_worker_grad_grouped(const float* X, const int32_t* y,
+                                 const float* W, const int32_t* offsets,
+                                 int32_t K, int32_t D, int32_t C,
+                                 float* const* G, float* losses,
+                                 void* workspace, size_t workspace_bytes,
+                                 void* cuda_stream);
+
+size_t db_worker_grad_grouped_workspace_bytes(int32_t total_rows, int32_t K,
+                                              int32_t D, int32_t C);
+
+/* ------------------------------------------------------------------------
  * The dense fp32 contraction db_worker_grad is built from (both Z = X W and
  * G = X^T E are instances), exposed so that it can be checked in isolation:
  *     out(m, n) = sum_{k < K} A(m, k) * B(n, k)

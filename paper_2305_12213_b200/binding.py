@@ -51,6 +51,9 @@ _SIGNATURES = {
                                  c_void_p, c_void_p, c_size_t, c_void_p]),
     "db_worker_grad_ex": (c_int32, [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p,
                                     c_void_p, c_void_p, c_size_t, ctypes.c_uint32, c_void_p]),
+    "db_worker_grad_grouped": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32,
+                                         c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+    "db_worker_grad_grouped_workspace_bytes": (c_size_t, [c_int32, c_int32, c_int32, c_int32]),
     "db_contract_f32": (c_int32, [c_void_p, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p, c_int64,
                                   c_int64, c_int32, c_int32, c_int32, c_void_p, c_void_p]),
     "db_worker_grad_workspace_bytes": (c_size_t, [c_int32, c_int32, c_int32]),
@@ -243,6 +246,30 @@ def worker_grad(X: torch.Tensor, y: torch.Tensor, W: torch.Tensor, G: torch.Tens
         None if workspace is None else workspace.data_ptr(),
         0 if workspace is None else workspace.numel() * workspace.element_size(),
         int(flags), _stream_ptr(stream)))
+
+
+def worker_grad_grouped_workspace_bytes(total_rows: int, K: int, D: int, C: int) -> int:
+    return int(lib().db_worker_grad_grouped_workspace_bytes(int(total_rows), int(K), int(D), int(C)))
+
+
+def worker_grad_grouped(X: torch.Tensor, y: torch.Tensor, W: torch.Tensor, offsets: Sequence[int],
+                        G: Sequence[torch.Tensor], losses: Optional[torch.Tensor], workspace: torch.Tensor,
+                        stream: Optional[torch.cuda.Stream] = None) -> None:
+    """db_worker_grad_grouped: every worker's gradient (rows offsets[w]:offsets[w+1] of X, y) in three launches."""
+    K = len(G)
+    rows, D = X.shape
+    D2, C = W.shape
+    if len(offsets) != K + 1 or D2 != D or y.numel() != rows or int(offsets[-1]) != rows:
+        raise ValueError("shape mismatch")
+    for g in G:
+        if tuple(g.shape) != (D, C):
+            raise ValueError("G[w] must be [D, C]")
+    table = (c_void_p * K)(*[_dev_ptr(g, torch.float32, "G[w]") for g in G])
+    _check(lib().db_worker_grad_grouped(
+        _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.int32, "y"), _dev_ptr(W, torch.float32, "W"),
+        ctypes.cast(_i32_array(offsets), c_void_p), K, D, C, ctypes.cast(table, c_void_p),
+        _dev_ptr(losses, torch.float32, "losses"), workspace.data_ptr(),
+        workspace.numel() * workspace.element_size(), _stream_ptr(stream)))
 
 
 def contract_f32(A: torch.Tensor, B: torch.Tensor, out: torch.Tensor, status: torch.Tensor,

@@ -26,6 +26,8 @@
 
 #include <cstdint>
 
+#include "dynbatch.h"
+
 namespace dynbatch {
 namespace tc {
 
@@ -305,8 +307,7 @@ struct SmemLayout {
 // n_acc shorter ones that the epilogue adds with ordinary rounded fp32 additions.  The cross terms
 // are 2^-11 of the main one: the rounding of their own chain is invisible.
 template <int N_TILE, int MODE_A, int MODE_B>
-__global__ void __launch_bounds__(kThreads)
-tf32x3_gemm_kernel(const __grid_constant__ GemmArgs g) {
+__device__ __forceinline__ void tf32x3_gemm_body(const GemmArgs& g, const int split) {
     using L = SmemLayout<N_TILE>;
     constexpr int kStagePitch = N_TILE + 4;   // floats per row of the output staging tile (16-byte rows, no bank conflicts)
     static_assert(kTileM * kStagePitch * 4 <= kStages * L::kStage, "output staging fits in the operand stages");
@@ -322,7 +323,7 @@ tf32x3_gemm_kernel(const __grid_constant__ GemmArgs g) {
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int m0 = blockIdx.y * kTileM, n0 = blockIdx.x * N_TILE;
-    const int k_begin = blockIdx.z * g.k_per_split;
+    const int k_begin = split * g.k_per_split;
     const int k_end = min(g.K, k_begin + g.k_per_split);
     const int nkb = (k_end - k_begin + kBlockK - 1) / kBlockK;
 
@@ -388,7 +389,7 @@ tf32x3_gemm_kernel(const __grid_constant__ GemmArgs g) {
             const int quarter = warp & 3;
             const int m = m0 + quarter * 32 + lane;         // this thread's accumulator lane = output row
             const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-            float* obase = g.out + static_cast<long long>(blockIdx.z) * g.o_split + static_cast<long long>(m) * g.o_m;
+            float* obase = g.out + static_cast<long long>(split) * g.o_split + static_cast<long long>(m) * g.o_m;
             const int used = min(g.n_acc, nkb);
 #pragma unroll 1
             for (int c0 = (warp >> 2) * 32; c0 < N_TILE; c0 += 32 * (kLoaderWarps / 4)) {
@@ -435,7 +436,7 @@ tf32x3_gemm_kernel(const __grid_constant__ GemmArgs g) {
             asm volatile("bar.sync 1, %0;" ::"n"(kLoaderThreads) : "memory");
             if (alive) {
                 const float* stage = reinterpret_cast<const float*>(tiles);
-                float* obase = g.out + static_cast<long long>(blockIdx.z) * g.o_split;
+                float* obase = g.out + static_cast<long long>(split) * g.o_split;
                 const int rows = min(kTileM, g.M - m0), cols = min(N_TILE, g.N - n0);
                 constexpr int kVecPerRow = N_TILE / 4;                 // float4 per tile row
                 constexpr int kRowsPerPass = kLoaderThreads / kVecPerRow;
@@ -495,6 +496,36 @@ tf32x3_gemm_kernel(const __grid_constant__ GemmArgs g) {
         tc_fence_after();
         tmem_dealloc(tmem_base, tmem_cols);
     }
+}
+
+// One problem, blockIdx.z = split of the reduction.
+template <int N_TILE, int MODE_A, int MODE_B>
+__global__ void __launch_bounds__(kThreads)
+tf32x3_gemm_kernel(const __grid_constant__ GemmArgs g) {
+    tf32x3_gemm_body<N_TILE, MODE_A, MODE_B>(g, blockIdx.z);
+}
+
+// Several problems that share every stride, M and N but have their own operands, output and
+// reduction length (the ragged per-worker gradients): blockIdx.z = problem, no split.
+struct GroupArgs {
+    const float* A[DB_MAX_K];
+    const float* B[DB_MAX_K];
+    float* out[DB_MAX_K];
+    int K[DB_MAX_K];
+};
+
+template <int N_TILE, int MODE_A, int MODE_B>
+__global__ void __launch_bounds__(kThreads)
+tf32x3_gemm_grouped_kernel(const __grid_constant__ GemmArgs shared, const __grid_constant__ GroupArgs groups) {
+    GemmArgs g = shared;
+    const int z = blockIdx.z;
+    g.A = groups.A[z];
+    g.B = groups.B[z];
+    g.out = groups.out[z];
+    g.K = groups.K[z];
+    g.k_per_split = (g.K + kBlockK - 1) / kBlockK * kBlockK;
+    if (g.k_per_split == 0) g.k_per_split = kBlockK;
+    tf32x3_gemm_body<N_TILE, MODE_A, MODE_B>(g, 0);
 }
 
 }  // namespace tc

@@ -156,15 +156,27 @@ __device__ __forceinline__ float block_reduce(float x, float* smem, bool take_ma
 // order comes from an atomic ticket (zeroed by the caller), nobody waits.
 // IN_REGS: C <= 4 * kThreads, every thread keeps its four logits in registers (one pass over memory);
 // otherwise the logits are parked in E between the passes.
+// Rows [off[w], off[w + 1]) belong to worker w; each worker has its own 1/b, ticket and loss slot.
+struct RowGroups {
+    int K;
+    int off[DB_MAX_K + 1];
+};
+
 template <bool IN_REGS>
 __global__ void __launch_bounds__(kThreads)
 softmax_residual_kernel(const float* __restrict__ partials, int splits, long long split_stride,
                         const int32_t* __restrict__ y, float* __restrict__ E, float* __restrict__ row_loss,
-                        int b, int C, unsigned int* __restrict__ ticket, float* __restrict__ loss) {
+                        const __grid_constant__ RowGroups groups, int C, unsigned int* __restrict__ tickets,
+                        float* __restrict__ losses) {
     __shared__ float smem[kThreads / 32];
     __shared__ float z_label;
     __shared__ bool is_last;
     const int i = blockIdx.x;
+    int w = 0;
+    while (w + 1 < groups.K && i >= groups.off[w + 1]) ++w;
+    const int row0 = groups.off[w], b = groups.off[w + 1] - row0;
+    unsigned int* ticket = tickets + w;
+    float* loss = losses ? losses + w : nullptr;
     float* e = E + static_cast<long long>(i) * C;
     const float* z0 = partials + static_cast<long long>(i) * C;
     const int label = y[i];
@@ -243,15 +255,26 @@ softmax_residual_kernel(const float* __restrict__ partials, int splits, long lon
     if (loss == nullptr) return;
     if (threadIdx.x == 0) {
         __threadfence();
-        is_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+        is_last = atomicAdd(ticket, 1u) == static_cast<unsigned int>(b) - 1u;
     }
     __syncthreads();
     if (!is_last) return;
     __threadfence();
     float part = 0.0f;
-    for (int r = threadIdx.x; r < b; r += kThreads) part += __ldcg(row_loss + r);
+    for (int r = threadIdx.x; r < b; r += kThreads) part += __ldcg(row_loss + row0 + r);
     const float total = block_reduce(part, smem, false);
     if (threadIdx.x == 0) *loss = total * inv_b;
+}
+
+void launch_softmax(const float* partials, int splits, long long split_stride, const int32_t* y, float* E,
+                    float* row_loss, const RowGroups& groups, int rows, int C, unsigned int* tickets, float* losses,
+                    cudaStream_t stream) {
+    if (C <= 4 * kThreads)
+        softmax_residual_kernel<true><<<rows, kThreads, 0, stream>>>(partials, splits, split_stride, y, E, row_loss,
+                                                                     groups, C, tickets, losses);
+    else
+        softmax_residual_kernel<false><<<rows, kThreads, 0, stream>>>(partials, splits, split_stride, y, E, row_loss,
+                                                                      groups, C, tickets, losses);
 }
 
 size_t round16(size_t x) { return (x + 15) & ~static_cast<size_t>(15); }
@@ -309,22 +332,32 @@ WorkerLayout layout_for(int b, int D, int C, bool tensor) {
 bool valid_shape(int b, int D, int C) { return b >= 1 && b <= 65535 && D >= 1 && C >= 1; }
 
 using TcKernel = void (*)(const tc::GemmArgs);
+using TcGroupedKernel = void (*)(const tc::GemmArgs, const tc::GroupArgs);
 
 template <int N_TILE, int MODE_A>
-TcKernel pick_tc_b(int mode_b) {
+void pick_tc_b(int mode_b, TcKernel* single, TcGroupedKernel* grouped) {
     switch (mode_b) {
-        case tc::kLoadKVec: return tc::tf32x3_gemm_kernel<N_TILE, MODE_A, tc::kLoadKVec>;
-        case tc::kLoadRowVec: return tc::tf32x3_gemm_kernel<N_TILE, MODE_A, tc::kLoadRowVec>;
-        default: return tc::tf32x3_gemm_kernel<N_TILE, MODE_A, tc::kLoadScalar>;
+        case tc::kLoadKVec:
+            *single = tc::tf32x3_gemm_kernel<N_TILE, MODE_A, tc::kLoadKVec>;
+            *grouped = tc::tf32x3_gemm_grouped_kernel<N_TILE, MODE_A, tc::kLoadKVec>;
+            break;
+        case tc::kLoadRowVec:
+            *single = tc::tf32x3_gemm_kernel<N_TILE, MODE_A, tc::kLoadRowVec>;
+            *grouped = tc::tf32x3_gemm_grouped_kernel<N_TILE, MODE_A, tc::kLoadRowVec>;
+            break;
+        default:
+            *single = tc::tf32x3_gemm_kernel<N_TILE, MODE_A, tc::kLoadScalar>;
+            *grouped = tc::tf32x3_gemm_grouped_kernel<N_TILE, MODE_A, tc::kLoadScalar>;
+            break;
     }
 }
 
 template <int N_TILE>
-TcKernel pick_tc(int mode_a, int mode_b) {
+void pick_tc(int mode_a, int mode_b, TcKernel* single, TcGroupedKernel* grouped) {
     switch (mode_a) {
-        case tc::kLoadKVec: return pick_tc_b<N_TILE, tc::kLoadKVec>(mode_b);
-        case tc::kLoadRowVec: return pick_tc_b<N_TILE, tc::kLoadRowVec>(mode_b);
-        default: return pick_tc_b<N_TILE, tc::kLoadScalar>(mode_b);
+        case tc::kLoadKVec: pick_tc_b<N_TILE, tc::kLoadKVec>(mode_b, single, grouped); break;
+        case tc::kLoadRowVec: pick_tc_b<N_TILE, tc::kLoadRowVec>(mode_b, single, grouped); break;
+        default: pick_tc_b<N_TILE, tc::kLoadScalar>(mode_b, single, grouped); break;
     }
 }
 
@@ -336,26 +369,51 @@ int load_mode(const float* p, long long row_stride, long long k_stride) {
     return tc::kLoadScalar;
 }
 
+int weaker_mode(int a, int b) { return a == b ? a : tc::kLoadScalar; }
+
 // out(m, n) = sum_k A(m, k) B(n, k) on the tensor cores; a.k_per_split must be a multiple of 32.
-db_status launch_tc_gemm(tc::GemmArgs a, int n_tile, cudaStream_t stream) {
+// With `groups` (n_groups problems sharing strides, M and N) blockIdx.z selects the problem.
+db_status launch_tc_gemm(tc::GemmArgs a, int n_tile, cudaStream_t stream, const tc::GroupArgs* groups = nullptr,
+                         int n_groups = 0) {
     if (n_tile != 32 && n_tile != 64) n_tile = 128;
+    int mode_a, mode_b, max_k = a.K;
+    if (groups) {
+        mode_a = load_mode(groups->A[0], a.a_row, a.a_k);
+        mode_b = load_mode(groups->B[0], a.b_row, a.b_k);
+        max_k = 0;
+        for (int z = 0; z < n_groups; ++z) {
+            mode_a = weaker_mode(mode_a, load_mode(groups->A[z], a.a_row, a.a_k));
+            mode_b = weaker_mode(mode_b, load_mode(groups->B[z], a.b_row, a.b_k));
+            if (groups->K[z] > max_k) max_k = groups->K[z];
+        }
+        a.k_per_split = (max_k + tc::kBlockK - 1) / tc::kBlockK * tc::kBlockK;
+    } else {
+        mode_a = load_mode(a.A, a.a_row, a.a_k);
+        mode_b = load_mode(a.B, a.b_row, a.b_k);
+    }
     // one main accumulator per four reduction blocks (chains of 16 additions), within 512 columns
     const int blocks = a.k_per_split / tc::kBlockK;
     int n_acc = (blocks + 3) / 4;
     if (n_acc > 512 / n_tile - 1) n_acc = 512 / n_tile - 1;
     a.n_acc = n_acc < 1 ? 1 : n_acc;
-    const int mode_a = load_mode(a.A, a.a_row, a.a_k), mode_b = load_mode(a.B, a.b_row, a.b_k);
-    TcKernel fn;
+    TcKernel fn = nullptr;
+    TcGroupedKernel gfn = nullptr;
     int smem;
     switch (n_tile) {
-        case 32: fn = pick_tc<32>(mode_a, mode_b); smem = tc::SmemLayout<32>::kBytes; break;
-        case 64: fn = pick_tc<64>(mode_a, mode_b); smem = tc::SmemLayout<64>::kBytes; break;
-        default: fn = pick_tc<128>(mode_a, mode_b); smem = tc::SmemLayout<128>::kBytes; n_tile = 128; break;
+        case 32: pick_tc<32>(mode_a, mode_b, &fn, &gfn); smem = tc::SmemLayout<32>::kBytes; break;
+        case 64: pick_tc<64>(mode_a, mode_b, &fn, &gfn); smem = tc::SmemLayout<64>::kBytes; break;
+        default: pick_tc<128>(mode_a, mode_b, &fn, &gfn); smem = tc::SmemLayout<128>::kBytes; break;
     }
-    DB_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    const int splits = a.k_per_split > 0 ? (a.K + a.k_per_split - 1) / a.k_per_split : 1;
-    dim3 grid((a.N + n_tile - 1) / n_tile, (a.M + tc::kTileM - 1) / tc::kTileM, splits < 1 ? 1 : splits);
-    fn<<<grid, tc::kThreads, smem, stream>>>(a);
+    if (groups) {
+        DB_CUDA_TRY(cudaFuncSetAttribute(gfn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        dim3 grid((a.N + n_tile - 1) / n_tile, (a.M + tc::kTileM - 1) / tc::kTileM, n_groups);
+        gfn<<<grid, tc::kThreads, smem, stream>>>(a, *groups);
+    } else {
+        DB_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        const int splits = a.k_per_split > 0 ? (a.K + a.k_per_split - 1) / a.k_per_split : 1;
+        dim3 grid((a.N + n_tile - 1) / n_tile, (a.M + tc::kTileM - 1) / tc::kTileM, splits < 1 ? 1 : splits);
+        fn<<<grid, tc::kThreads, smem, stream>>>(a);
+    }
     DB_CUDA_TRY(cudaGetLastError());
     return DB_OK;
 }
@@ -434,12 +492,12 @@ extern "C" db_status db_worker_grad_ex(const float* X, const int32_t* y, const f
         DB_CUDA_TRY(cudaGetLastError());
     }
     // 2. softmax residual (P - Y) / b
-    if (C <= 4 * kThreads)
-        softmax_residual_kernel<true><<<b_i, kThreads, 0, stream>>>(partials, L.splits, bc, y, E, row_loss, b_i, C,
-                                                                    reinterpret_cast<unsigned int*>(status) + 1, loss);
-    else
-        softmax_residual_kernel<false><<<b_i, kThreads, 0, stream>>>(partials, L.splits, bc, y, E, row_loss, b_i, C,
-                                                                     reinterpret_cast<unsigned int*>(status) + 1, loss);
+    RowGroups one{};
+    one.K = 1;
+    one.off[0] = 0;
+    one.off[1] = b_i;
+    launch_softmax(partials, L.splits, bc, y, E, row_loss, one, b_i, C, reinterpret_cast<unsigned int*>(status) + 1,
+                   loss, stream);
     DB_CUDA_TRY(cudaGetLastError());
     // 3. G = X^T E
     if (tensor) {
@@ -460,6 +518,113 @@ extern "C" db_status db_worker_grad_ex(const float* X, const int32_t* y, const f
         else
             tile_gemm_kernel<true, false><<<grid, kThreads, 0, stream>>>(X, D, E, C, G, C, 0, D, C, b_i, b_i);
         DB_CUDA_TRY(cudaGetLastError());
+    }
+    return DB_OK;
+}
+
+namespace dynbatch {
+namespace {
+
+struct GroupedLayout {
+    int splits, k_per_split, n_tile;
+    size_t header_bytes, partial_bytes, e_bytes, loss_bytes;
+    size_t total() const { return header_bytes + partial_bytes + e_bytes + loss_bytes; }
+};
+
+// All workers' rows go through one logits contraction (they share W); split over D for about one CTA per SM.
+GroupedLayout grouped_layout(long long rows, int K, int D, int C) {
+    GroupedLayout L;
+    L.n_tile = rows <= 32 ? 32 : (rows <= 64 ? 64 : 128);
+    const long long tiles = static_cast<long long>((C + tc::kTileM - 1) / tc::kTileM) * ((rows + L.n_tile - 1) / L.n_tile);
+    long long s = sm_count() / tiles;
+    const int kblocks = (D + tc::kBlockK - 1) / tc::kBlockK;
+    if (s > kblocks) s = kblocks;
+    if (s < 1) s = 1;
+    const int per_blocks = static_cast<int>((kblocks + s - 1) / s);
+    L.k_per_split = per_blocks * tc::kBlockK;
+    L.splits = (D + L.k_per_split - 1) / L.k_per_split;
+    L.header_bytes = round16(kStatusBytes + sizeof(unsigned int) * static_cast<size_t>(K));
+    L.partial_bytes = round16(sizeof(float) * static_cast<size_t>(L.splits) * rows * C);
+    L.e_bytes = round16(sizeof(float) * static_cast<size_t>(rows) * C);
+    L.loss_bytes = round16(sizeof(float) * static_cast<size_t>(rows));
+    return L;
+}
+
+bool valid_group_shape(long long rows, int K, int D, int C) {
+    return K >= 1 && K <= DB_MAX_K && rows >= K && rows <= (1 << 22) && D >= 1 && C >= 1;
+}
+
+}  // namespace
+}  // namespace dynbatch
+
+extern "C" size_t db_worker_grad_grouped_workspace_bytes(int32_t total_rows, int32_t K, int32_t D, int32_t C) {
+    using namespace dynbatch;
+    if (!valid_group_shape(total_rows, K, D, C)) return 0;
+    return grouped_layout(total_rows, K, D, C).total();
+}
+
+extern "C" db_status db_worker_grad_grouped(const float* X, const int32_t* y, const float* W,
+                                            const int32_t* offsets, int32_t K, int32_t D, int32_t C,
+                                            float* const* G, float* losses, void* workspace,
+                                            size_t workspace_bytes, void* cuda_stream) {
+    using namespace dynbatch;
+    if (!X || !y || !W || !offsets || !G || !workspace) return DB_ERR_NULL;
+    if (K < 1 || K > DB_MAX_K || D < 1 || C < 1) return DB_ERR_ARG;
+    if (offsets[0] != 0) return DB_ERR_ARG;
+    for (int w = 0; w < K; ++w) {
+        const long long bw = static_cast<long long>(offsets[w + 1]) - offsets[w];
+        if (bw < 1) return DB_ERR_ARG;                         // every worker holds at least one sample
+        if (bw > kMaxTensorCoreBatch) return DB_ERR_UNSUPPORTED;
+        if (!G[w]) return DB_ERR_NULL;
+    }
+    const long long rows = offsets[K];
+    if (!valid_group_shape(rows, K, D, C)) return DB_ERR_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) % 16) return DB_ERR_ARG;
+    const GroupedLayout L = grouped_layout(rows, K, D, C);
+    if (workspace_bytes < L.total()) return DB_ERR_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    char* base = static_cast<char*>(workspace);
+    int* status = reinterpret_cast<int*>(base);
+    unsigned int* tickets = reinterpret_cast<unsigned int*>(base + kStatusBytes);
+    float* partials = reinterpret_cast<float*>(base + L.header_bytes);
+    float* E = reinterpret_cast<float*>(base + L.header_bytes + L.partial_bytes);
+    float* row_loss = reinterpret_cast<float*>(base + L.header_bytes + L.partial_bytes + L.e_bytes);
+    const long long rc = rows * C;
+    DB_CUDA_TRY(cudaMemsetAsync(base, 0, L.header_bytes, stream));
+
+    // 1. logits of every row, transposed orientation, split over D
+    {
+        tc::GemmArgs a{};
+        a.A = W; a.a_row = 1; a.a_k = C;
+        a.B = X; a.b_row = D; a.b_k = 1;
+        a.out = partials; a.o_m = 1; a.o_n = C; a.o_split = rc;
+        a.M = C; a.N = static_cast<int>(rows); a.K = D; a.k_per_split = L.k_per_split; a.status = status;
+        const db_status st = launch_tc_gemm(a, L.n_tile, stream);
+        if (st != DB_OK) return st;
+    }
+    // 2. softmax residual with each worker's own 1/b
+    RowGroups rg{};
+    rg.K = K;
+    for (int w = 0; w <= K; ++w) rg.off[w] = offsets[w];
+    launch_softmax(partials, L.splits, rc, y, E, row_loss, rg, static_cast<int>(rows), C, tickets, losses, stream);
+    DB_CUDA_TRY(cudaGetLastError());
+    // 3. one gradient per worker: G_w = X_w^T E_w, reduction over that worker's rows only
+    {
+        tc::GemmArgs a{};
+        a.a_row = 1; a.a_k = D;
+        a.b_row = 1; a.b_k = C;
+        a.o_m = C; a.o_n = 1; a.o_split = 0;
+        a.M = D; a.N = C; a.status = status;
+        tc::GroupArgs gr{};
+        for (int w = 0; w < K; ++w) {
+            gr.A[w] = X + static_cast<long long>(offsets[w]) * D;
+            gr.B[w] = E + static_cast<long long>(offsets[w]) * C;
+            gr.out[w] = G[w];
+            gr.K[w] = offsets[w + 1] - offsets[w];
+        }
+        const db_status st = launch_tc_gemm(a, 64, stream, &gr, K);
+        if (st != DB_OK) return st;
     }
     return DB_OK;
 }

@@ -101,3 +101,54 @@ def test_config_ragged_four_workers_against_the_concatenated_batch(flags):
     # the uniform average of the four gradients is a different vector
     uniform = torch.stack(Gs).double().mean(0).cpu().numpy()
     assert rel_err(uniform, full) > 1e-2
+
+
+# ------------------------------------------------------------------ grouped (all workers in three launches)
+def _grouped(X, y, W, bs):
+    offs = [0] + list(np.cumsum(bs))
+    D, C = W.shape
+    G = [torch.full((D, C), float("nan"), device=DEV) for _ in bs]
+    losses = torch.zeros(len(bs), device=DEV)
+    ws = torch.empty(binding.worker_grad_grouped_workspace_bytes(offs[-1], len(bs), D, C), dtype=torch.uint8,
+                     device=DEV)
+    binding.worker_grad_grouped(X, y, W, offs, G, losses, ws)
+    torch.cuda.synchronize()
+    assert binding.worker_grad_status(ws) == 0
+    return G, losses.cpu().numpy(), offs
+
+
+@pytest.mark.parametrize("bs,D,C", [([24, 40, 64, 128], 2048, 1000), ([1], 8, 4), ([1, 1, 1], 33, 10),
+                                     ([5, 130, 2, 33, 70], 100, 130), ([300, 7], 64, 1030)])
+def test_grouped_matches_the_oracle_per_worker(bs, D, C):
+    X, y, W = inputs.softmax_problem(bs, D, C, seed=4000 + len(bs), w_std=0.02, device=DEV)
+    G, losses, offs = _grouped(X, y, W, bs)
+    Xh, yh, Wh = X.cpu().numpy(), y.cpu().numpy(), W.cpu().numpy()
+    for w in range(len(bs)):
+        rG, rloss = oracle.worker_grad(Xh[offs[w]:offs[w + 1]], yh[offs[w]:offs[w + 1]], Wh)
+        assert rel_err(f64(G[w]), rG) <= FP32_TOL, f"worker {w}"
+        assert abs(losses[w] - rloss) <= FP32_TOL * abs(rloss)
+
+
+def test_grouped_then_aggregate_is_the_concatenated_batch_gradient():
+    bs = [24, 40, 64, 128]
+    D, C = 2048, 1000
+    X, y, W = inputs.softmax_problem(bs, D, C, seed=3000, device=DEV)
+    G, _, _ = _grouped(X, y, W, bs)
+    N = D * C
+    p, v = torch.zeros(N, device=DEV), torch.zeros(N, device=DEV)
+    binding.aggregate_update([g.reshape(-1) for g in G], bs, p, v, 1.0, 0.0)
+    torch.cuda.synchronize()
+    full, _ = oracle.worker_grad(X.cpu().numpy(), y.cpu().numpy(), W.cpu().numpy())
+    assert rel_err(f64(v), full.reshape(-1)) <= FP32_TOL
+
+
+def test_grouped_argument_errors():
+    X, y, W = inputs.softmax_problem([4, 4], 16, 8, seed=9, device=DEV)
+    G = [torch.empty(16, 8, device=DEV) for _ in range(2)]
+    ws = torch.empty(binding.worker_grad_grouped_workspace_bytes(8, 2, 16, 8), dtype=torch.uint8, device=DEV)
+    for offs in ([0, 4, 4], [1, 4, 8], [0, 5, 4]):           # empty worker, bad start, decreasing
+        Xs = X[:max(offs[-1], 1)]
+        with pytest.raises((binding.DynbatchError, ValueError)):
+            binding.worker_grad_grouped(X[:offs[-1]], y[:offs[-1]], W, offs, G, None, ws)
+    with pytest.raises(binding.DynbatchError):
+        binding.worker_grad_grouped(X, y, W, [0, 4, 8], G, None, ws[:64])
