@@ -113,7 +113,7 @@ size_t db_aggregate_workspace_bytes(int32_t K, int64_t N);
  * cudaMalloc is forbidden because it may synchronise the whole device; code
  * that only ever receives raw input/output pointers from its framework.  For
  * them this entry point keeps the scratch inside the library, in a fixed
- * array in device global memory (DB_STATIC_SCRATCH_BYTES, resident on every
+ * array in device global memory (DB_STATIC_SCRATCH_BYTES = 1 MiB, resident on every
  * GPU that loads the library until the process exits).  It calls no
  * cudaMalloc/cudaFree and no allocating library routine.
  *
@@ -129,12 +129,13 @@ size_t db_aggregate_workspace_bytes(int32_t K, int64_t N);
  *     whose kernels may run at the same time on one device (different
  *     streams, different threads) race on it and return a wrong norm:
  *     serialise them, or use db_aggregate_update_ex with separate workspaces.
- *   - If the scratch this device needs (db_aggregate_workspace_bytes) exceeds
- *     DB_STATIC_SCRATCH_BYTES the call returns DB_ERR_UNSUPPORTED and enqueues
- *     nothing; db_last_cuda_error() then says how many bytes were needed.
- *     N itself is not limited: the scratch grows with the GPU's SM count only.
+ *   - The scratch holds one double per CTA, i.e. per 1024 parameters, so the
+ *     built-in 1 MiB serves N up to 134,182,912 parameters when the norm is
+ *     requested (any N without it).  Beyond that the call returns
+ *     DB_ERR_UNSUPPORTED and enqueues nothing; db_last_cuda_error() then says
+ *     how many bytes were needed.
  * ------------------------------------------------------------------------ */
-#define DB_STATIC_SCRATCH_BYTES 65536
+#define DB_STATIC_SCRATCH_BYTES 1048576
 
 db_status db_aggregate_update_static(const void* const* grads,
                                      db_dtype grad_dtype, const int32_t* b,
@@ -325,6 +326,57 @@ db_status db_controller_step(int32_t* b, const double* throughputs, int32_t K,
 db_status db_controller_step_ex(int32_t* b, const double* throughputs,
                                 int32_t K, double kp, const int32_t* b_min,
                                 const int32_t* b_max);
+
+/* ------------------------------------------------------------------------
+ * Static open-loop allocation                               (Section 3.2)
+ *
+ * b_k proportional to the throughput estimate X_k with the global batch K*b0
+ * kept: b_k = K * b0 * X_k / sum X (the printed b0 * X_k / sum X sums to b0,
+ * not to the K*b0 the text requires), made integer within the bounds by the
+ * same largest-remainder rule as the controller.
+ *   throughputs host, K finite values > 0 (e.g. core counts or FLOPs)
+ *   b0          the uniform per-worker batch it replaces, >= 1
+ *   b_min,b_max host, K each, or NULL for 1 and K*b0
+ *   b           host, K, written on DB_OK
+ * ------------------------------------------------------------------------ */
+db_status db_static_allocate(const double* throughputs, int32_t K, int32_t b0,
+                             const int32_t* b_min, const int32_t* b_max,
+                             int32_t* b);
+
+/* ------------------------------------------------------------------------
+ * Stabilised controller, host side        (Section 3.3.1, the 4-step listing)
+ *
+ * A controller object keeps the current batch sizes and, per observation of
+ * the workers' iteration times t_k (any unit, > 0):
+ *   1. smooths them with an EWMA over the iterations since the last
+ *      readjustment, mu_k <- alpha t_k + (1 - alpha) mu_k (the first sample
+ *      after a readjustment initialises mu_k; the paper gives no alpha);
+ *   2. applies db_controller_step_ex with X_k = b_k / mu_k and gain kp;
+ *   3. within [b_min, b_max]; with adaptive_b_max != 0 the upper bound also
+ *      learns: when a worker whose batch was raised at the previous
+ *      readjustment (from b0 to b) now shows a lower smoothed throughput than
+ *      it had then, its upper bound becomes b0.  If the learnt bounds cannot
+ *      hold the global batch, the user's bounds alone are used for that step;
+ *   4. dead-band: the new sizes are adopted for all workers only if
+ *      max_k |b'_k - b_k| / b_k > dead_band (the paper uses 0.05), else none.
+ *
+ *   b0          host, K initial batch sizes >= 1
+ *   kp          0 < kp <= 1;  alpha 0 < alpha <= 1;  dead_band >= 0
+ *   b_min,b_max host, K each, or NULL for 1 and sum(b0)
+ * db_controller_observe: b_out (host, K, nullable) receives the batch sizes in
+ * force after the observation, *changed (nullable) whether they moved.
+ * Not thread-safe per object.  All arithmetic is IEEE fp64 in a fixed order.
+ * ------------------------------------------------------------------------ */
+typedef struct db_controller db_controller;
+
+db_status db_controller_create(db_controller** out, const int32_t* b0,
+                               int32_t K, double kp, double alpha,
+                               double dead_band, const int32_t* b_min,
+                               const int32_t* b_max, int32_t adaptive_b_max);
+db_status db_controller_observe(db_controller* controller,
+                                const double* iteration_times, int32_t* b_out,
+                                int32_t* changed);
+db_status db_controller_destroy(db_controller* controller);
 
 /* Static text for a status code. */
 const char* db_status_string(db_status s);

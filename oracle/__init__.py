@@ -41,7 +41,8 @@ def lib():
             c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]
         L.ref_controller_observe.argtypes = [
             c_void_p, c_void_p, c_int32, c_double, c_double, c_double,
-            c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+            c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int32,
+            c_void_p, c_void_p, c_void_p]
         L.ref_num_threads.restype = ctypes.c_int
         L.ref_set_num_threads.argtypes = [ctypes.c_int]
         _lib = L
@@ -174,8 +175,12 @@ def static_allocate(X, b0, b_min=None, b_max=None):
 class ControllerState:
     """State of the stabilised controller: batch sizes, EWMA, samples since readjust."""
 
-    def __init__(self, b, kp=1.0, alpha=0.5, dmin=0.05, b_min=None, b_max=None):
+    def __init__(self, b, kp=1.0, alpha=0.5, dmin=0.05, b_min=None, b_max=None, adaptive=False):
+        self.adaptive = bool(adaptive)
         self.b = _i32(b).copy()
+        self.prev_b = np.zeros(self.b.size, dtype=np.int32)
+        self.prev_X = np.zeros(self.b.size, dtype=np.float64)
+        self.learnt_max = np.zeros(self.b.size, dtype=np.int32)
         self.kp, self.alpha, self.dmin = float(kp), float(alpha), float(dmin)
         self.lo = None if b_min is None else _i32(b_min)
         self.hi = None if b_max is None else _i32(b_max)
@@ -188,7 +193,8 @@ class ControllerState:
         _check(lib().ref_controller_observe(
             _ptr(self.b), _ptr(t), self.b.size, self.kp, self.alpha, self.dmin,
             _ptr(self.lo), _ptr(self.hi), _ptr(self.ewma), _ptr(self.n_since),
-            _ptr(changed)))
+            _ptr(changed), int(self.adaptive), _ptr(self.prev_b), _ptr(self.prev_X),
+            _ptr(self.learnt_max)))
         return bool(changed[0])
 
 

@@ -354,17 +354,27 @@ int ref_static_allocate(const double* X, int32_t K, int32_t b0,
  *      weight of the new sample -- the paper gives no value);
  *   2. Eq. 4-5 with mu_k in place of t_k (X_k = b_k / mu_k), gain kp,
  *      rescaled to the global batch, made integer within the bounds;
- *   3. bounds b_min <= b <= b_max (inside the apportionment);
+ *   3. bounds b_min <= b <= b_max (inside the apportionment).  With
+ *      `adaptive` set, the upper bound also learns ("Batch size bounds"): if
+ *      a worker's smoothed throughput is lower than it was at the previous
+ *      readjustment although its batch was raised then (from b0 to b), its
+ *      upper bound becomes b0.  Should the learnt bounds no longer admit the
+ *      global batch, the user's bounds alone are used for this step;
  *   4. dead-band: readjust every worker only if max_k |b'_k - b_k| / b_k
  *      exceeds dmin (the paper uses 0.05), else keep all batch sizes.
- * State: ewma[K], n_since (samples since the last readjustment, 0 = none).
- * *changed is set to 1 when the batch sizes were readjusted.
+ * State: ewma[K], n_since (samples since the last readjustment, 0 = none),
+ * and for the adaptive bound prev_b[K], prev_X[K] (batch and throughput at
+ * the previous readjustment; prev_X = 0 means none yet) and learnt_max[K]
+ * (0 = nothing learnt).  *changed is set to 1 when the batch sizes moved.
  */
 int ref_controller_observe(int32_t* b, const double* t, int32_t K, double kp,
                            double alpha, double dmin, const int32_t* b_min,
                            const int32_t* b_max, double* ewma,
-                           int32_t* n_since, int32_t* changed) {
+                           int32_t* n_since, int32_t* changed,
+                           int32_t adaptive, int32_t* prev_b, double* prev_X,
+                           int32_t* learnt_max) {
     if (!b || !t || !ewma || !n_since || !changed || K < 1) return REF_ERR_ARG;
+    if (adaptive && (!prev_b || !prev_X || !learnt_max)) return REF_ERR_ARG;
     if (!(alpha > 0.0) || !(alpha <= 1.0) || !(dmin >= 0.0)) return REF_ERR_ARG;
     for (int32_t k = 0; k < K; ++k)
         if (!(t[k] > 0.0) || !isfinite(t[k]) || b[k] < 1) return REF_ERR_ARG;
@@ -373,9 +383,29 @@ int ref_controller_observe(int32_t* b, const double* t, int32_t K, double kp,
     *n_since += 1;
     double* X = (double*)malloc(sizeof(double) * (size_t)K);
     int32_t* nb = (int32_t*)malloc(sizeof(int32_t) * (size_t)K);
-    if (!X || !nb) { free(X); free(nb); return REF_ERR_ARG; }
-    for (int32_t k = 0; k < K; ++k) { X[k] = (double)b[k] / ewma[k]; nb[k] = b[k]; }
-    int rc = ref_controller_step(nb, X, K, kp, b_min, b_max);
+    int32_t* hi = (int32_t*)malloc(sizeof(int32_t) * (size_t)K);
+    if (!X || !nb || !hi) { free(X); free(nb); free(hi); return REF_ERR_ARG; }
+    int64_t S = 0;
+    for (int32_t k = 0; k < K; ++k) { X[k] = (double)b[k] / ewma[k]; nb[k] = b[k]; S += b[k]; }
+    int use_learnt = 0;
+    if (adaptive) {
+        for (int32_t k = 0; k < K; ++k) {
+            if (prev_X[k] > 0.0 && b[k] > prev_b[k] && X[k] < prev_X[k]) {
+                if (learnt_max[k] == 0 || prev_b[k] < learnt_max[k]) learnt_max[k] = prev_b[k];
+            }
+        }
+        for (int32_t k = 0; k < K; ++k) {
+            int64_t h = b_max ? b_max[k] : S;
+            if (learnt_max[k] > 0 && learnt_max[k] < h) { h = learnt_max[k]; use_learnt = 1; }
+            hi[k] = (int32_t)h;
+        }
+    }
+    int rc = REF_ERR_INFEASIBLE;
+    if (use_learnt) rc = ref_controller_step(nb, X, K, kp, b_min, hi);
+    if (rc == REF_ERR_INFEASIBLE) {
+        for (int32_t k = 0; k < K; ++k) nb[k] = b[k];
+        rc = ref_controller_step(nb, X, K, kp, b_min, b_max);
+    }
     *changed = 0;
     if (rc == REF_OK) {
         double worst = 0.0;
@@ -384,6 +414,8 @@ int ref_controller_observe(int32_t* b, const double* t, int32_t K, double kp,
             if (rel > worst) worst = rel;
         }
         if (worst > dmin) {
+            if (adaptive)
+                for (int32_t k = 0; k < K; ++k) { prev_b[k] = b[k]; prev_X[k] = X[k]; }
             memcpy(b, nb, sizeof(int32_t) * (size_t)K);
             *n_since = 0;
             *changed = 1;
@@ -391,6 +423,7 @@ int ref_controller_observe(int32_t* b, const double* t, int32_t K, double kp,
     }
     free(X);
     free(nb);
+    free(hi);
     return rc;
 }
 

@@ -59,6 +59,11 @@ _SIGNATURES = {
     "db_worker_grad_workspace_bytes": (c_size_t, [c_int32, c_int32, c_int32]),
     "db_controller_step": (c_int32, [c_void_p, c_void_p, c_int32, c_double]),
     "db_controller_step_ex": (c_int32, [c_void_p, c_void_p, c_int32, c_double, c_void_p, c_void_p]),
+    "db_static_allocate": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]),
+    "db_controller_create": (c_int32, [c_void_p, c_void_p, c_int32, c_double, c_double, c_double, c_void_p,
+                                       c_void_p, c_int32]),
+    "db_controller_observe": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p]),
+    "db_controller_destroy": (c_int32, [c_void_p]),
     "db_status_string": (c_char_p, [c_int32]),
     "db_last_cuda_error": (c_char_p, []),
 }
@@ -306,3 +311,49 @@ def controller_step(b: Sequence[int], throughputs: Sequence[float], kp: float,
     _check(lib().db_controller_step_ex(ctypes.cast(arr, c_void_p), ctypes.cast(xs, c_void_p), K,
                                        float(kp), lo, hi))
     return list(arr)
+
+
+def static_allocate(throughputs: Sequence[float], b0: int, b_min: Optional[Sequence[int]] = None,
+                    b_max: Optional[Sequence[int]] = None) -> list:
+    """db_static_allocate: throughput-proportional batch sizes that keep the global batch K * b0."""
+    K = len(throughputs)
+    xs = (c_double * K)(*[float(x) for x in throughputs])
+    out = (c_int32 * K)()
+    lo = None if b_min is None else ctypes.cast(_i32_array(b_min), c_void_p)
+    hi = None if b_max is None else ctypes.cast(_i32_array(b_max), c_void_p)
+    _check(lib().db_static_allocate(ctypes.cast(xs, c_void_p), K, int(b0), lo, hi, ctypes.cast(out, c_void_p)))
+    return list(out)
+
+
+class Controller:
+    """db_controller: the stabilised batch-size controller (EWMA, bounds, dead-band)."""
+
+    def __init__(self, b0: Sequence[int], kp: float = 1.0, alpha: float = 0.5, dead_band: float = 0.05,
+                 b_min: Optional[Sequence[int]] = None, b_max: Optional[Sequence[int]] = None,
+                 adaptive_b_max: bool = False):
+        self.K = len(b0)
+        self._h = c_void_p()
+        lo = None if b_min is None else ctypes.cast(_i32_array(b_min), c_void_p)
+        hi = None if b_max is None else ctypes.cast(_i32_array(b_max), c_void_p)
+        _check(lib().db_controller_create(ctypes.byref(self._h), ctypes.cast(_i32_array(b0), c_void_p), self.K,
+                                          float(kp), float(alpha), float(dead_band), lo, hi, int(adaptive_b_max)))
+
+    def observe(self, iteration_times: Sequence[float]):
+        """Returns (batch sizes in force, whether they were readjusted)."""
+        ts = (c_double * self.K)(*[float(t) for t in iteration_times])
+        out = (c_int32 * self.K)()
+        changed = c_int32(0)
+        _check(lib().db_controller_observe(self._h, ctypes.cast(ts, c_void_p), ctypes.cast(out, c_void_p),
+                                           ctypes.byref(changed)))
+        return list(out), bool(changed.value)
+
+    def close(self) -> None:
+        if self._h:
+            lib().db_controller_destroy(self._h)
+            self._h = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -176,3 +176,68 @@ def test_controller_scenario_with_throughput_drop(lib):
         assert b_lib == b_ref.tolist() and sum(b_lib) == 512
     want = 512 * np.array(X) / sum(X)
     assert np.abs(np.array(b_lib) - want).max() <= 1.0
+
+
+# ------------------------------------------------------------------ static allocation and stabilised controller
+def test_static_allocate_matches_oracle_and_the_papers_clusters(lib):
+    assert binding.static_allocate([3, 9, 18], 100) == [30, 90, 180]
+    assert binding.static_allocate([0.813, 0.187], 500) == [813, 187]
+    rng = np.random.default_rng(11)
+    for trial in range(100):
+        K = int(rng.integers(1, 20))
+        X = rng.uniform(0.1, 30.0, size=K).tolist()
+        b0 = int(rng.integers(1, 200))
+        lo = [int(v) for v in rng.integers(0, b0 // 2 + 1, size=K)] if trial % 3 == 0 else None
+        hi = [int(v) for v in rng.integers(b0, 4 * b0 + 1, size=K)] if trial % 4 == 0 else None
+        try:
+            ref = oracle.static_allocate(X, b0, lo, hi).tolist()
+        except oracle.OracleError as e:
+            with pytest.raises(binding.DynbatchError) as ei:
+                binding.static_allocate(X, b0, lo, hi)
+            assert ei.value.status == e.code
+            continue
+        assert binding.static_allocate(X, b0, lo, hi) == ref
+    with pytest.raises(binding.DynbatchError):
+        binding.static_allocate([1.0, -1.0], 8)
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_stabilised_controller_bit_exact_against_oracle(lib, seed):
+    rng = np.random.default_rng(100 + seed)
+    K = int(rng.integers(2, 12))
+    b0 = [int(v) for v in rng.integers(8, 128, size=K)]
+    kp = float(rng.choice([0.5, 1.0]))
+    alpha = float(rng.choice([0.3, 0.5, 1.0]))
+    dmin = float(rng.choice([0.0, 0.05, 0.2]))
+    adaptive = bool(seed % 2)
+    lo = [int(v) for v in rng.integers(1, 8, size=K)] if seed % 3 == 0 else None
+    hi = [int(v) for v in rng.integers(128, 512, size=K)] if seed % 5 == 0 else None
+    X = rng.uniform(0.5, 8.0, size=K)
+    cliff = rng.integers(64, 256, size=K)                   # throughput halves above this batch
+    ref = oracle.ControllerState(b0, kp, alpha, dmin, lo, hi, adaptive)
+    ctl = binding.Controller(b0, kp, alpha, dmin, lo, hi, adaptive)
+    b = list(b0)
+    for it in range(60):
+        if it == 30:
+            X[0] *= 0.5
+        eff = np.where(np.array(b) > cliff, 0.5 * X, X)
+        t = (np.array(b) / eff * (1.0 + 0.02 * rng.standard_normal(K))).tolist()
+        changed_ref = ref.observe(t)
+        b, changed = ctl.observe(t)
+        assert b == ref.b.tolist() and changed == changed_ref, f"iteration {it}"
+        assert sum(b) == sum(b0)
+    ctl.close()
+
+
+def test_stabilised_controller_argument_errors(lib):
+    E = binding
+    with pytest.raises(E.DynbatchError):
+        E.Controller([0, 4])
+    with pytest.raises(E.DynbatchError):
+        E.Controller([4, 4], alpha=0.0)
+    with pytest.raises(E.DynbatchError):
+        E.Controller([4, 4], dead_band=-1.0)
+    c = E.Controller([4, 4])
+    with pytest.raises(E.DynbatchError):
+        c.observe([1.0, 0.0])
+    assert c.observe([1.0, 1.0]) == ([4, 4], False)

@@ -447,3 +447,27 @@ def test_dead_band_stops_oscillation_under_noise():
         moves[dmin] = n
         assert st.b.sum() == 192
     assert moves[0.05] == 0 and moves[0.0] > 0
+
+
+def test_adaptive_upper_bound_learns_from_a_throughput_drop():
+    """Fig. 5 / "Batch size bounds": worker 0's throughput collapses above a batch of 100 (memory limit).
+    Without learning the controller keeps pushing it over the cliff; with it the bound b_max = the last
+    good batch is learnt and the batch stays at or below it."""
+    def times(b):
+        X0 = 10.0 if b[0] <= 100 else 4.0
+        return [b[0] / X0, b[1] / 2.0]
+
+    st = oracle.ControllerState([64, 64], kp=1.0, alpha=1.0, dmin=0.0, adaptive=True)
+    history = []
+    for _ in range(8):
+        st.observe(times(st.b))
+        history.append(int(st.b[0]))
+    assert history[0] > 100                      # first adjustment overshoots the cliff (10:2 split of 128)
+    assert int(st.learnt_max[0]) == 64           # the drop is seen: back to the last batch that ran well
+    assert max(history[2:]) <= 64 and st.b.sum() == 128
+    plain = oracle.ControllerState([64, 64], kp=1.0, alpha=1.0, dmin=0.0, adaptive=False)
+    seen = []
+    for _ in range(8):
+        plain.observe(times(plain.b))
+        seen.append(int(plain.b[0]))
+    assert max(seen[2:]) > 100                   # without the learnt bound it keeps crossing the cliff
