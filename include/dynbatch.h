@@ -103,6 +103,28 @@ db_status db_aggregate_update_ex(const void* const* grads, db_dtype grad_dtype,
 size_t db_aggregate_workspace_bytes(int32_t K, int64_t N);
 
 /* ------------------------------------------------------------------------
+ * Weighted aggregation + Adam update   (Section 3.1, Eq. 2; Adam is the
+ * optimizer of the paper's MNIST workload, Section 4, which prints no formula:
+ * this is the textbook rule with bias correction)
+ *
+ * Same aggregate g as above, then per parameter, with t = step >= 1:
+ *     m <- beta1 m + (1 - beta1) g        u <- beta2 u + (1 - beta2) g^2
+ *     p <- p - lr * (m / (1 - beta1^t)) / (sqrt(u / (1 - beta2^t)) + eps)
+ * first_moment and second_moment are device fp32 buffers of N elements updated
+ * in place (zero before step 1).  0 <= beta1, beta2 < 1, eps >= 0.  Every other
+ * argument, the alignment rules, the norm and the workspace are those of
+ * db_aggregate_update_ex; the pass reads K gradients + 3 state arrays and
+ * writes 3: K * sizeof(grad) + 24 bytes per parameter.
+ * ------------------------------------------------------------------------ */
+db_status db_aggregate_adam_ex(const void* const* grads, db_dtype grad_dtype,
+                               const int32_t* b, int32_t K, int64_t N,
+                               float* params, float* first_moment,
+                               float* second_moment, float lr, float beta1,
+                               float beta2, float eps, int64_t step,
+                               double* grad_sqnorm, void* workspace,
+                               size_t workspace_bytes, void* cuda_stream);
+
+/* ------------------------------------------------------------------------
  * The same step for callers that cannot provide scratch memory
  * (the paper has no counterpart; this is a packaging variant of the call above)
  *

@@ -39,6 +39,9 @@ _SIGNATURES = {
                                          c_void_p, c_float, c_float, c_void_p, c_void_p, c_size_t,
                                          c_void_p]),
     "db_aggregate_workspace_bytes": (c_size_t, [c_int32, c_int64]),
+    "db_aggregate_adam_ex": (c_int32, [c_void_p, c_int32, c_void_p, c_int32, c_int64, c_void_p, c_void_p, c_void_p,
+                                       c_float, c_float, c_float, c_float, c_int64, c_void_p, c_void_p, c_size_t,
+                                       c_void_p]),
     "db_aggregate_update_static": (c_int32, [c_void_p, c_int32, c_void_p, c_int32, c_int64, c_void_p,
                                              c_void_p, c_float, c_float, c_void_p, c_void_p]),
     "db_host_pipeline_create": (c_int32, [c_void_p]),
@@ -147,6 +150,27 @@ def aggregate_update(grads: Sequence[torch.Tensor], b: Sequence[int], params: to
         None if workspace is None else workspace.data_ptr(),
         0 if workspace is None else workspace.numel() * workspace.element_size(),
         _stream_ptr(stream)))
+
+
+def aggregate_adam(grads: Sequence[torch.Tensor], b: Sequence[int], params: torch.Tensor,
+                   first_moment: torch.Tensor, second_moment: torch.Tensor, lr: float, beta1: float,
+                   beta2: float, eps: float, step: int, grad_sqnorm: Optional[torch.Tensor] = None,
+                   workspace: Optional[torch.Tensor] = None,
+                   stream: Optional[torch.cuda.Stream] = None) -> None:
+    """db_aggregate_adam_ex: fused weighted aggregation + Adam update (bias-corrected), in place."""
+    K = len(grads)
+    if len(b) != K:
+        raise ValueError("len(b) != len(grads)")
+    gdt = grads[0].dtype
+    table = (c_void_p * K)(*[_dev_ptr(g, gdt, "grads[k]") for g in grads])
+    code = DB_F32 if gdt == torch.float32 else DB_BF16 if gdt == torch.bfloat16 else -1
+    _check(lib().db_aggregate_adam_ex(
+        ctypes.cast(table, c_void_p), code, ctypes.cast(_i32_array(b), c_void_p), K, int(params.numel()),
+        _dev_ptr(params, torch.float32, "params"), _dev_ptr(first_moment, torch.float32, "first_moment"),
+        _dev_ptr(second_moment, torch.float32, "second_moment"), float(lr), float(beta1), float(beta2),
+        float(eps), int(step), _dev_ptr(grad_sqnorm, torch.float64, "grad_sqnorm"),
+        None if workspace is None else workspace.data_ptr(),
+        0 if workspace is None else workspace.numel() * workspace.element_size(), _stream_ptr(stream)))
 
 
 def aggregate_update_static(grads: Sequence[torch.Tensor], b: Sequence[int], params: torch.Tensor,

@@ -6,13 +6,14 @@
 // vectors before the first use, folds the slices with fp32 FMAs in worker
 // order, applies v = mu v + g, p = p - lr v and streams both back.  Nothing
 // else touches N-sized data; the squared gradient norm rides along in
-// registers.  One CTA handles one tile of 256 x UNROLL vectors and exits: the
-// hardware hands out tiles in index order as CTAs retire, which keeps all SMs
-// inside one narrow moving window of each stream.  Measured on B200 this beats a
-// persistent grid-stride grid of SMs x occupancy CTAs by 2-14 % (K = 16 .. 2):
-// persistent CTAs drift apart and spread the DRAM accesses over more pages.
+// registers.  A CTA handles one to four consecutive tiles of 256 x UNROLL vectors and
+// exits: the hardware hands out CTAs in index order as others retire, so the SMs
+// stay inside one narrow moving window of each stream and their load and store
+// phases are staggered.  Measured on B200 this beats a persistent grid-stride grid
+// of SMs x occupancy CTAs by 2-14 % (K = 16 .. 2), whose CTAs move in lock step.
 #include <cuda_bf16.h>
 
+#include <cmath>
 #include <cstdint>
 #include <cstdio>
 
@@ -29,16 +30,37 @@ struct AggArgs {
     const void* g[DB_MAX_K];  // active workers' gradient buffers
     float lambda[DB_MAX_K];   // their weights b_k / sum b
     float* p;
-    float* v;
+    float* v;                 // momentum (heavy ball) or first moment (Adam)
+    float* u;                 // second moment (Adam only)
     double* partials;         // one per CTA (norm only)
     unsigned int* ticket;     // CTA arrival counter, zero at launch (norm only)
     double* sq_out;
     long long n;              // elements
     long long head;           // leading elements before the first 16-byte boundary
     long long nvec;           // whole vectors after the head
-    float lr, mu;
+    float lr, mu;             // mu: momentum coefficient, or Adam's beta1
+    float beta2, eps, inv_c1, inv_c2;   // Adam: 1 / (1 - beta^t) bias corrections
     int K;
 };
+
+enum Optimizer { kMomentum = 0, kAdam = 1 };
+
+// The optimizer step on one element, given the aggregated gradient g.
+//   momentum: v <- mu v + g;                  p <- p - lr v
+//   Adam:     m <- b1 m + (1 - b1) g;  u <- b2 u + (1 - b2) g^2;
+//             p <- p - lr (m / c1) / (sqrt(u / c2) + eps)
+template <int OPT>
+__device__ __forceinline__ void optimizer_step(const AggArgs& a, float g, float& p, float& v, float& u) {
+    if (OPT == kMomentum) {
+        v = fmaf(a.mu, v, g);
+        p = fmaf(-a.lr, v, p);
+    } else {
+        v = fmaf(a.mu, v, (1.0f - a.mu) * g);
+        u = fmaf(a.beta2, u, (1.0f - a.beta2) * (g * g));
+        const float denom = sqrtf(u * a.inv_c2) + a.eps;
+        p = p - a.lr * (v * a.inv_c1) / denom;
+    }
+}
 
 // Raw 16-byte gradient vector and its widening to fp32 lanes.
 template <typename GT> struct GradVec;
@@ -115,37 +137,35 @@ __device__ __forceinline__ void finish_norm(const AggArgs& a, double sq) {
 }
 
 // One element, any alignment: the same FMA chain as the vector body.
-template <typename GT, bool NORM>
+template <typename GT, bool NORM, int OPT>
 __device__ __forceinline__ void update_scalar(const AggArgs& a, int K, long long j, double& sq) {
     float g = 0.0f;
     for (int k = 0; k < K; ++k) g = fmaf(a.lambda[k], GradVec<GT>::scalar(a.g[k], j), g);
-    const float vn = fmaf(a.mu, a.v[j], g);
-    a.v[j] = vn;
-    a.p[j] = fmaf(-a.lr, vn, a.p[j]);
+    float p = a.p[j], v = a.v[j], u = OPT == kAdam ? a.u[j] : 0.0f;
+    optimizer_step<OPT>(a, g, p, v, u);
+    a.v[j] = v;
+    a.p[j] = p;
+    if (OPT == kAdam) a.u[j] = u;
     if (NORM) sq += static_cast<double>(g * g);
 }
 
-// Momentum update of the `kLanes` elements at vector index vi.
-template <int kLanes, bool NORM>
+// Optimizer update of the `kLanes` elements at vector index vi.
+template <int kLanes, bool NORM, int OPT>
 __device__ __forceinline__ void apply_update(const AggArgs& a, long long vi, const float (&g)[kLanes],
-                                             const float4 (&pv)[kLanes / 4], const float4 (&vv)[kLanes / 4],
-                                             double& sq) {
+                                             float4 (&pv)[kLanes / 4], float4 (&vv)[kLanes / 4],
+                                             float4 (&uv)[kLanes / 4], double& sq) {
     float4* pp = reinterpret_cast<float4*>(a.p + a.head) + vi * (kLanes / 4);
     float4* vp = reinterpret_cast<float4*>(a.v + a.head) + vi * (kLanes / 4);
     float part = 0.0f;
 #pragma unroll
     for (int q = 0; q < kLanes / 4; ++q) {
-        float4 vn, pn;
-        vn.x = fmaf(a.mu, vv[q].x, g[4 * q + 0]);
-        vn.y = fmaf(a.mu, vv[q].y, g[4 * q + 1]);
-        vn.z = fmaf(a.mu, vv[q].z, g[4 * q + 2]);
-        vn.w = fmaf(a.mu, vv[q].w, g[4 * q + 3]);
-        pn.x = fmaf(-a.lr, vn.x, pv[q].x);
-        pn.y = fmaf(-a.lr, vn.y, pv[q].y);
-        pn.z = fmaf(-a.lr, vn.z, pv[q].z);
-        pn.w = fmaf(-a.lr, vn.w, pv[q].w);
-        __stcs(vp + q, vn);
-        __stcs(pp + q, pn);
+        optimizer_step<OPT>(a, g[4 * q + 0], pv[q].x, vv[q].x, uv[q].x);
+        optimizer_step<OPT>(a, g[4 * q + 1], pv[q].y, vv[q].y, uv[q].y);
+        optimizer_step<OPT>(a, g[4 * q + 2], pv[q].z, vv[q].z, uv[q].z);
+        optimizer_step<OPT>(a, g[4 * q + 3], pv[q].w, vv[q].w, uv[q].w);
+        __stcs(vp + q, vv[q]);
+        __stcs(pp + q, pv[q]);
+        if (OPT == kAdam) __stcs(reinterpret_cast<float4*>(a.u + a.head) + vi * (kLanes / 4) + q, uv[q]);
         if (NORM) {
 #pragma unroll
             for (int l = 0; l < 4; ++l) part = fmaf(g[4 * q + l], g[4 * q + l], part);
@@ -155,7 +175,8 @@ __device__ __forceinline__ void apply_update(const AggArgs& a, long long vi, con
 }
 
 // KT > 0: exactly KT workers, fully unrolled.  KT == 0: a.K workers, kChunk at a time.
-template <typename GT, int KT, int UNROLL, bool NORM>
+// A CTA handles TILES consecutive tiles of kBlock x UNROLL vectors.
+template <typename GT, int KT, int UNROLL, int TILES, bool NORM, int OPT>
 __global__ void __launch_bounds__(kBlock)
 agg_vec_kernel(const __grid_constant__ AggArgs a) {
     using GV = GradVec<GT>;
@@ -166,11 +187,13 @@ agg_vec_kernel(const __grid_constant__ AggArgs a) {
     double sq = 0.0;
 
     const long long tile = static_cast<long long>(kBlock) * UNROLL;
-    const long long base = static_cast<long long>(blockIdx.x) * tile;   // one tile per CTA
-    if (base < a.nvec) {
+#pragma unroll 1
+    for (int t = 0; t < TILES; ++t) {
+        const long long base = (static_cast<long long>(blockIdx.x) * TILES + t) * tile;
+        if (base >= a.nvec) break;
         long long vi[UNROLL];
         bool ok[UNROLL];
-        float4 pv[UNROLL][kQuads], vv[UNROLL][kQuads];
+        float4 pv[UNROLL][kQuads], vv[UNROLL][kQuads], uv[UNROLL][kQuads];
         float g[UNROLL][kLanes];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
@@ -190,6 +213,8 @@ agg_vec_kernel(const __grid_constant__ AggArgs a) {
                 for (int q = 0; q < kQuads; ++q) {
                     pv[u][q] = __ldcs(reinterpret_cast<const float4*>(a.p + a.head) + vi[u] * kQuads + q);
                     vv[u][q] = __ldcs(reinterpret_cast<const float4*>(a.v + a.head) + vi[u] * kQuads + q);
+                    if (OPT == kAdam)
+                        uv[u][q] = __ldcs(reinterpret_cast<const float4*>(a.u + a.head) + vi[u] * kQuads + q);
                 }
             }
 #pragma unroll
@@ -211,6 +236,8 @@ agg_vec_kernel(const __grid_constant__ AggArgs a) {
                 for (int q = 0; q < kQuads; ++q) {
                     pv[u][q] = __ldcs(reinterpret_cast<const float4*>(a.p + a.head) + vi[u] * kQuads + q);
                     vv[u][q] = __ldcs(reinterpret_cast<const float4*>(a.v + a.head) + vi[u] * kQuads + q);
+                    if (OPT == kAdam)
+                        uv[u][q] = __ldcs(reinterpret_cast<const float4*>(a.u + a.head) + vi[u] * kQuads + q);
                 }
                 for (int k0 = 0; k0 < K; k0 += kChunk) {
                     Raw raw[kChunk];
@@ -232,26 +259,26 @@ agg_vec_kernel(const __grid_constant__ AggArgs a) {
         }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u)
-            if (ok[u]) apply_update<kLanes, NORM>(a, vi[u], g[u], pv[u], vv[u], sq);
+            if (ok[u]) apply_update<kLanes, NORM, OPT>(a, vi[u], g[u], pv[u], vv[u], uv[u], sq);
     }
 
     // ragged ends: fewer than kLanes elements on either side of the vector body
     if (blockIdx.x == 0) {
         const long long tail0 = a.head + a.nvec * kLanes;
-        if (threadIdx.x < a.head) update_scalar<GT, NORM>(a, K, threadIdx.x, sq);
-        if (tail0 + threadIdx.x < a.n) update_scalar<GT, NORM>(a, K, tail0 + threadIdx.x, sq);
+        if (threadIdx.x < a.head) update_scalar<GT, NORM, OPT>(a, K, threadIdx.x, sq);
+        if (tail0 + threadIdx.x < a.n) update_scalar<GT, NORM, OPT>(a, K, tail0 + threadIdx.x, sq);
     }
     if (NORM) finish_norm(a, sq);
 }
 
 // Element-wise kernel for buffers whose 16-byte boundaries do not line up.
-template <typename GT, bool NORM>
+template <typename GT, bool NORM, int OPT>
 __global__ void __launch_bounds__(kBlock)
 agg_scalar_kernel(const __grid_constant__ AggArgs a) {
     double sq = 0.0;
     const long long step = static_cast<long long>(gridDim.x) * kBlock;
     for (long long j = static_cast<long long>(blockIdx.x) * kBlock + threadIdx.x; j < a.n; j += step)
-        update_scalar<GT, NORM>(a, a.K, j, sq);
+        update_scalar<GT, NORM, OPT>(a, a.K, j, sq);
     if (NORM) finish_norm(a, sq);
 }
 
@@ -262,23 +289,26 @@ constexpr size_t kTicketBytes = 256;  // ticket word, padded so the partials sta
 
 using KernelFn = void (*)(const AggArgs);
 
-template <typename GT, int KT, bool NORM>
-KernelFn pick_unroll(int* unroll_out) {
-    // two vector positions per thread: 2 (K + 2) independent 16-byte loads in flight; measured best or
-    // within 0.5 % of best for K = 2 .. 16 (four positions spill at K = 16)
-    constexpr int kUnroll = KT > 0 ? 2 : 1;
-    *unroll_out = kUnroll;
-    return agg_vec_kernel<GT, KT, kUnroll, NORM>;
+template <typename GT, int KT, bool NORM, int OPT>
+KernelFn pick_unroll(int* vectors_per_cta) {
+    // Measured on B200 (with the norm): up to 8 workers, two vector positions per thread and one tile
+    // per CTA (2 (K + 2) independent 16-byte loads in flight per thread); 9 to 16 workers, one position
+    // per thread (registers) and two consecutive tiles per CTA, which amortises the norm epilogue;
+    // the chunked many-worker kernel one tile (more tiles per CTA cost it 30 %).
+    constexpr int kUnroll = (KT >= 1 && KT <= 8) ? 2 : 1;
+    constexpr int kTiles = (KT >= 9) ? 2 : 1;
+    *vectors_per_cta = kBlock * kUnroll * kTiles;
+    return agg_vec_kernel<GT, KT, kUnroll, kTiles, NORM, OPT>;
 }
 
-template <typename GT, bool NORM>
+template <typename GT, bool NORM, int OPT>
 KernelFn pick_vec_kernel(int K, int* unroll_out) {
     switch (K) {
-#define DB_CASE(n) case n: return pick_unroll<GT, n, NORM>(unroll_out);
+#define DB_CASE(n) case n: return pick_unroll<GT, n, NORM, OPT>(unroll_out);
         DB_CASE(1) DB_CASE(2) DB_CASE(3) DB_CASE(4) DB_CASE(5) DB_CASE(6) DB_CASE(7) DB_CASE(8)
         DB_CASE(9) DB_CASE(10) DB_CASE(11) DB_CASE(12) DB_CASE(13) DB_CASE(14) DB_CASE(15) DB_CASE(16)
 #undef DB_CASE
-        default: return pick_unroll<GT, 0, NORM>(unroll_out);
+        default: return pick_unroll<GT, 0, NORM, OPT>(unroll_out);
     }
 }
 
@@ -312,16 +342,30 @@ extern "C" size_t db_aggregate_workspace_bytes(int32_t K, int64_t N) {
     return dynbatch::kTicketBytes + sizeof(double) * static_cast<size_t>(dynbatch::cta_bound(N < 0 ? 0 : N));
 }
 
-extern "C" db_status db_aggregate_update_ex(const void* const* grads, db_dtype grad_dtype,
-                                            const int32_t* b, int32_t K, int64_t N,
-                                            float* params, float* momentum, float lr, float mu,
-                                            double* grad_sqnorm, void* workspace,
-                                            size_t workspace_bytes, void* cuda_stream) {
-    using namespace dynbatch;
+namespace dynbatch {
+namespace {
+
+template <int OPT>
+KernelFn pick_kernel(bool vector_ok, db_dtype dt, bool norm, int active, int* vectors_per_cta) {
+    if (vector_ok) {
+        if (dt == DB_F32)
+            return norm ? pick_vec_kernel<float, true, OPT>(active, vectors_per_cta)
+                        : pick_vec_kernel<float, false, OPT>(active, vectors_per_cta);
+        return norm ? pick_vec_kernel<__nv_bfloat16, true, OPT>(active, vectors_per_cta)
+                    : pick_vec_kernel<__nv_bfloat16, false, OPT>(active, vectors_per_cta);
+    }
+    if (dt == DB_F32) return norm ? agg_scalar_kernel<float, true, OPT> : agg_scalar_kernel<float, false, OPT>;
+    return norm ? agg_scalar_kernel<__nv_bfloat16, true, OPT> : agg_scalar_kernel<__nv_bfloat16, false, OPT>;
+}
+
+// Validation, weights, alignment analysis and launch shared by the momentum and Adam entry points.
+// `a` arrives with the optimizer's scalars set; `second` is Adam's second-moment buffer (else NULL).
+db_status aggregate_launch(AggArgs a, int opt, const void* const* grads, db_dtype grad_dtype, const int32_t* b,
+                           int32_t K, int64_t N, float* params, float* first, float* second,
+                           double* grad_sqnorm, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     if (!grads || !b) return DB_ERR_NULL;
     if (K < 1 || K > DB_MAX_K || N < 0) return DB_ERR_ARG;
     if (grad_dtype != DB_F32 && grad_dtype != DB_BF16) return DB_ERR_UNSUPPORTED;
-    if (!isfinite(lr) || !isfinite(mu)) return DB_ERR_ARG;
     long long total = 0;
     for (int k = 0; k < K; ++k) {
         if (b[k] < 0) return DB_ERR_ARG;
@@ -329,31 +373,33 @@ extern "C" db_status db_aggregate_update_ex(const void* const* grads, db_dtype g
     }
     if (total <= 0) return DB_ERR_ARG;
     if (N == 0) return DB_OK;
-    if (!params || !momentum) return DB_ERR_NULL;
+    float* state[3] = {params, first, second};
+    const int n_state = opt == kAdam ? 3 : 2;
     const size_t gsize = grad_dtype == DB_F32 ? 4 : 2;
     const size_t state_bytes = static_cast<size_t>(N) * 4, grad_bytes = static_cast<size_t>(N) * gsize;
-    if (reinterpret_cast<uintptr_t>(params) % 4 || reinterpret_cast<uintptr_t>(momentum) % 4) return DB_ERR_ARG;
-    if (ranges_overlap(params, state_bytes, momentum, state_bytes)) return DB_ERR_ARG;
+    for (int i = 0; i < n_state; ++i) {
+        if (!state[i]) return DB_ERR_NULL;
+        if (reinterpret_cast<uintptr_t>(state[i]) % 4) return DB_ERR_ARG;
+        for (int j = 0; j < i; ++j)
+            if (ranges_overlap(state[i], state_bytes, state[j], state_bytes)) return DB_ERR_ARG;
+    }
 
-    AggArgs a{};
     int active = 0;
     for (int k = 0; k < K; ++k) {
         if (b[k] == 0) continue;  // weight 0: the buffer is not read
         if (!grads[k]) return DB_ERR_NULL;
         if (reinterpret_cast<uintptr_t>(grads[k]) % gsize) return DB_ERR_ARG;
-        if (ranges_overlap(grads[k], grad_bytes, params, state_bytes) ||
-            ranges_overlap(grads[k], grad_bytes, momentum, state_bytes))
-            return DB_ERR_ARG;
+        for (int i = 0; i < n_state; ++i)
+            if (ranges_overlap(grads[k], grad_bytes, state[i], state_bytes)) return DB_ERR_ARG;
         a.g[active] = grads[k];
         a.lambda[active] = static_cast<float>(static_cast<double>(b[k]) / static_cast<double>(total));
         ++active;
     }
     a.K = active;
     a.p = params;
-    a.v = momentum;
+    a.v = first;
+    a.u = second;
     a.n = N;
-    a.lr = lr;
-    a.mu = mu;
 
     const bool norm = grad_sqnorm != nullptr;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -366,11 +412,13 @@ extern "C" db_status db_aggregate_update_ex(const void* const* grads, db_dtype g
         a.sq_out = grad_sqnorm;
     }
 
-    // Leading elements until params reaches a 16-byte boundary; the vector body
-    // needs momentum and every gradient buffer on a boundary at the same element.
+    // Leading elements until params reaches a 16-byte boundary; the vector body needs the other
+    // state buffers and every gradient buffer on a boundary at the same element.
     const int lanes = grad_dtype == DB_F32 ? 4 : 8;
     long long head = static_cast<long long>(((16 - reinterpret_cast<uintptr_t>(params) % 16) % 16) / 4);
-    bool vector_ok = (reinterpret_cast<uintptr_t>(momentum) + head * 4) % 16 == 0;
+    bool vector_ok = true;
+    for (int i = 1; i < n_state; ++i)
+        vector_ok = vector_ok && (reinterpret_cast<uintptr_t>(state[i]) + head * 4) % 16 == 0;
     if (vector_ok && grad_dtype == DB_BF16) {
         // bf16 vectors hold 8 elements: pick the head in {head, head + 4} that aligns the gradients
         const uintptr_t g0 = reinterpret_cast<uintptr_t>(a.g[0]);
@@ -382,30 +430,58 @@ extern "C" db_status db_aggregate_update_ex(const void* const* grads, db_dtype g
     a.head = head;
     a.nvec = (N - head) / lanes;
 
-    KernelFn fn;
+    int vectors_per_cta = kBlock;
+    const KernelFn fn = opt == kAdam ? pick_kernel<kAdam>(vector_ok, grad_dtype, norm, active, &vectors_per_cta)
+                                     : pick_kernel<kMomentum>(vector_ok, grad_dtype, norm, active, &vectors_per_cta);
     int grid;
     if (vector_ok) {
-        int unroll = 1;
-        if (grad_dtype == DB_F32)
-            fn = norm ? pick_vec_kernel<float, true>(active, &unroll) : pick_vec_kernel<float, false>(active, &unroll);
-        else
-            fn = norm ? pick_vec_kernel<__nv_bfloat16, true>(active, &unroll)
-                      : pick_vec_kernel<__nv_bfloat16, false>(active, &unroll);
-        const long long tile = static_cast<long long>(kBlock) * unroll;
-        const long long tiles = (a.nvec + tile - 1) / tile;
+        const long long tiles = (a.nvec + vectors_per_cta - 1) / vectors_per_cta;
         if (tiles > 0x7fffffffLL) return DB_ERR_ARG;
         grid = static_cast<int>(tiles < 1 ? 1 : tiles);
     } else {
-        if (grad_dtype == DB_F32)
-            fn = norm ? agg_scalar_kernel<float, true> : agg_scalar_kernel<float, false>;
-        else
-            fn = norm ? agg_scalar_kernel<__nv_bfloat16, true> : agg_scalar_kernel<__nv_bfloat16, false>;
         grid = scalar_grid(fn, N);
     }
     if (norm) DB_CUDA_TRY(cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), stream));
     fn<<<grid, kBlock, 0, stream>>>(a);
     DB_CUDA_TRY(cudaGetLastError());
     return DB_OK;
+}
+
+}  // namespace
+}  // namespace dynbatch
+
+extern "C" db_status db_aggregate_update_ex(const void* const* grads, db_dtype grad_dtype,
+                                            const int32_t* b, int32_t K, int64_t N,
+                                            float* params, float* momentum, float lr, float mu,
+                                            double* grad_sqnorm, void* workspace,
+                                            size_t workspace_bytes, void* cuda_stream) {
+    using namespace dynbatch;
+    if (!isfinite(lr) || !isfinite(mu)) return DB_ERR_ARG;
+    AggArgs a{};
+    a.lr = lr;
+    a.mu = mu;
+    return aggregate_launch(a, kMomentum, grads, grad_dtype, b, K, N, params, momentum, nullptr, grad_sqnorm,
+                            workspace, workspace_bytes, cuda_stream);
+}
+
+extern "C" db_status db_aggregate_adam_ex(const void* const* grads, db_dtype grad_dtype, const int32_t* b,
+                                          int32_t K, int64_t N, float* params, float* first_moment,
+                                          float* second_moment, float lr, float beta1, float beta2, float eps,
+                                          int64_t step, double* grad_sqnorm, void* workspace,
+                                          size_t workspace_bytes, void* cuda_stream) {
+    using namespace dynbatch;
+    if (!isfinite(lr) || !isfinite(eps) || !(eps >= 0.0f)) return DB_ERR_ARG;
+    if (!(beta1 >= 0.0f) || !(beta1 < 1.0f) || !(beta2 >= 0.0f) || !(beta2 < 1.0f) || step < 1) return DB_ERR_ARG;
+    AggArgs a{};
+    a.lr = lr;
+    a.mu = beta1;
+    a.beta2 = beta2;
+    a.eps = eps;
+    // bias corrections in fp64 on the host, once per call
+    a.inv_c1 = static_cast<float>(1.0 / (1.0 - pow(static_cast<double>(beta1), static_cast<double>(step))));
+    a.inv_c2 = static_cast<float>(1.0 / (1.0 - pow(static_cast<double>(beta2), static_cast<double>(step))));
+    return aggregate_launch(a, kAdam, grads, grad_dtype, b, K, N, params, first_moment, second_moment,
+                            grad_sqnorm, workspace, workspace_bytes, cuda_stream);
 }
 
 extern "C" db_status db_aggregate_update(const float* const* grads, const int32_t* b, int32_t K,
