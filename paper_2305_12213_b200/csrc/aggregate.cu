@@ -23,7 +23,6 @@ namespace dynbatch {
 namespace {
 
 constexpr int kBlock = 256;
-constexpr int kMaxFixedK = 16;   // K up to here gets a fully unrolled kernel
 constexpr int kChunk = 8;        // gradient slices loaded per round beyond that
 
 struct AggArgs {
@@ -530,7 +529,7 @@ extern "C" db_status db_aggregate_update_static(const void* const* grads, db_dty
     if (grad_sqnorm) {
         const size_t need = db_aggregate_workspace_bytes(K, N);
         if (need > DB_STATIC_SCRATCH_BYTES) {
-            char msg[160];
+            char msg[256];
             snprintf(msg, sizeof msg,
                      "db_aggregate_update_static: this device needs %zu bytes of scratch, the built-in "
                      "array holds %d; use db_aggregate_update_ex with a workspace",

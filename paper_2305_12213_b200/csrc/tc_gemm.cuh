@@ -92,6 +92,12 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         }
     }
 }
+// Programmatic dependent launch: let the next kernel in the stream start its prologue while this one
+// runs, and wait for the previous kernel's results before touching them.  Both are no-ops for a
+// kernel launched without the attribute.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -342,6 +348,9 @@ __device__ __forceinline__ void tf32x3_gemm_body(const GemmArgs& g, const int sp
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
+    // everything above overlaps the previous kernel; its outputs are read only from here on
+    griddep_launch_dependents();
+    griddep_wait();
 
     if (warp < kLoaderWarps) {
         // ------------------------------------------------------------ producers

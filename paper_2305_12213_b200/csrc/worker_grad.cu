@@ -3,11 +3,12 @@
 // the model on which Eq. 2's batch-proportional weights are checked against
 // the gradient of the concatenated global batch (Section 3.1).
 //
-// Three launches on the caller's stream:
+// A memset node (status word and tickets) and three launches on the caller's stream:
 //   1. logits: split over the feature dimension D so that a worker with a
 //      handful of rows still fills the GPU; partial sums go to the workspace;
 //   2. softmax: one CTA per sample folds the partials in split order, applies
 //      the max-subtracted softmax, subtracts the one-hot label, scales by 1/b_i;
+//      the last CTA of a worker also folds the per-sample losses into the mean;
 //   3. gradient: G = X^T E, reduction depth b_i.
 // The two contractions run on the tensor cores (tcgen05, three TF32 products per
 // fp32 product, see tc_gemm.cuh).  An fp32 FFMA version on shared-memory tiles is
@@ -171,6 +172,7 @@ softmax_residual_kernel(const float* __restrict__ partials, int splits, long lon
     __shared__ float smem[kThreads / 32];
     __shared__ float z_label;
     __shared__ bool is_last;
+    tc::griddep_launch_dependents();
     const int i = blockIdx.x;
     int w = 0;
     while (w + 1 < groups.K && i >= groups.off[w + 1]) ++w;
@@ -184,6 +186,7 @@ softmax_residual_kernel(const float* __restrict__ partials, int splits, long lon
     float zmax = -INFINITY;
     float z[4] = {0.0f, 0.0f, 0.0f, 0.0f};
     if (threadIdx.x == 0) z_label = 0.0f;
+    tc::griddep_wait();      // the logits kernel has finished and its partial sums are visible
     // four classes per thread and eight splits per round: 32 independent loads in flight, adds in split order
     for (int cb = 0; cb < C; cb += 4 * kThreads) {
 #pragma unroll
@@ -266,15 +269,34 @@ softmax_residual_kernel(const float* __restrict__ partials, int splits, long lon
     if (threadIdx.x == 0) *loss = total * inv_b;
 }
 
-void launch_softmax(const float* partials, int splits, long long split_stride, const int32_t* y, float* E,
-                    float* row_loss, const RowGroups& groups, int rows, int C, unsigned int* tickets, float* losses,
-                    cudaStream_t stream) {
+// Launch configuration of a kernel that may start while its predecessor in the stream still runs
+// (it calls griddepcontrol.wait before reading the predecessor's output).
+struct OverlappedLaunch {
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1]{};
+    OverlappedLaunch(dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool overlap) {
+        cfg.gridDim = grid;
+        cfg.blockDim = block;
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = overlap ? 1 : 0;
+    }
+};
+
+db_status launch_softmax(const float* partials, int splits, long long split_stride, const int32_t* y, float* E,
+                         float* row_loss, const RowGroups& groups, int rows, int C, unsigned int* tickets,
+                         float* losses, cudaStream_t stream, bool overlap) {
+    OverlappedLaunch L(dim3(rows), dim3(kThreads), 0, stream, overlap);
     if (C <= 4 * kThreads)
-        softmax_residual_kernel<true><<<rows, kThreads, 0, stream>>>(partials, splits, split_stride, y, E, row_loss,
-                                                                     groups, C, tickets, losses);
+        DB_CUDA_TRY(cudaLaunchKernelEx(&L.cfg, softmax_residual_kernel<true>, partials, splits, split_stride, y, E,
+                                       row_loss, groups, C, tickets, losses));
     else
-        softmax_residual_kernel<false><<<rows, kThreads, 0, stream>>>(partials, splits, split_stride, y, E, row_loss,
-                                                                      groups, C, tickets, losses);
+        DB_CUDA_TRY(cudaLaunchKernelEx(&L.cfg, softmax_residual_kernel<false>, partials, splits, split_stride, y, E,
+                                       row_loss, groups, C, tickets, losses));
+    return DB_OK;
 }
 
 size_t round16(size_t x) { return (x + 15) & ~static_cast<size_t>(15); }
@@ -374,7 +396,7 @@ int weaker_mode(int a, int b) { return a == b ? a : tc::kLoadScalar; }
 // out(m, n) = sum_k A(m, k) B(n, k) on the tensor cores; a.k_per_split must be a multiple of 32.
 // With `groups` (n_groups problems sharing strides, M and N) blockIdx.z selects the problem.
 db_status launch_tc_gemm(tc::GemmArgs a, int n_tile, cudaStream_t stream, const tc::GroupArgs* groups = nullptr,
-                         int n_groups = 0) {
+                         int n_groups = 0, bool overlap = false) {
     if (n_tile != 32 && n_tile != 64) n_tile = 128;
     int mode_a, mode_b, max_k = a.K;
     if (groups) {
@@ -407,12 +429,14 @@ db_status launch_tc_gemm(tc::GemmArgs a, int n_tile, cudaStream_t stream, const 
     if (groups) {
         DB_CUDA_TRY(cudaFuncSetAttribute(gfn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         dim3 grid((a.N + n_tile - 1) / n_tile, (a.M + tc::kTileM - 1) / tc::kTileM, n_groups);
-        gfn<<<grid, tc::kThreads, smem, stream>>>(a, *groups);
+        OverlappedLaunch L(grid, dim3(tc::kThreads), smem, stream, overlap);
+        DB_CUDA_TRY(cudaLaunchKernelEx(&L.cfg, gfn, a, *groups));
     } else {
         DB_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         const int splits = a.k_per_split > 0 ? (a.K + a.k_per_split - 1) / a.k_per_split : 1;
         dim3 grid((a.N + n_tile - 1) / n_tile, (a.M + tc::kTileM - 1) / tc::kTileM, splits < 1 ? 1 : splits);
-        fn<<<grid, tc::kThreads, smem, stream>>>(a);
+        OverlappedLaunch L(grid, dim3(tc::kThreads), smem, stream, overlap);
+        DB_CUDA_TRY(cudaLaunchKernelEx(&L.cfg, fn, a));
     }
     DB_CUDA_TRY(cudaGetLastError());
     return DB_OK;
@@ -496,9 +520,12 @@ extern "C" db_status db_worker_grad_ex(const float* X, const int32_t* y, const f
     one.K = 1;
     one.off[0] = 0;
     one.off[1] = b_i;
-    launch_softmax(partials, L.splits, bc, y, E, row_loss, one, b_i, C, reinterpret_cast<unsigned int*>(status) + 1,
-                   loss, stream);
-    DB_CUDA_TRY(cudaGetLastError());
+    {
+        // after the tensor-core logits kernel the softmax may start early (it waits for the partials itself)
+        const db_status st = launch_softmax(partials, L.splits, bc, y, E, row_loss, one, b_i, C,
+                                            reinterpret_cast<unsigned int*>(status) + 1, loss, stream, tensor);
+        if (st != DB_OK) return st;
+    }
     // 3. G = X^T E
     if (tensor) {
         tc::GemmArgs a{};
@@ -508,7 +535,7 @@ extern "C" db_status db_worker_grad_ex(const float* X, const int32_t* y, const f
         a.M = D; a.N = C; a.K = b_i;
         a.k_per_split = (b_i + tc::kBlockK - 1) / tc::kBlockK * tc::kBlockK;   // one split
         a.status = status;
-        const db_status st = launch_tc_gemm(a, 64, stream);
+        const db_status st = launch_tc_gemm(a, 64, stream, nullptr, 0, true);
         if (st != DB_OK) return st;
     } else {
         const bool vec4 = (D % 4 == 0) && (C % 4 == 0) && aligned16(X) && aligned16(G);
@@ -607,8 +634,11 @@ extern "C" db_status db_worker_grad_grouped(const float* X, const int32_t* y, co
     RowGroups rg{};
     rg.K = K;
     for (int w = 0; w <= K; ++w) rg.off[w] = offsets[w];
-    launch_softmax(partials, L.splits, rc, y, E, row_loss, rg, static_cast<int>(rows), C, tickets, losses, stream);
-    DB_CUDA_TRY(cudaGetLastError());
+    {
+        const db_status st = launch_softmax(partials, L.splits, rc, y, E, row_loss, rg, static_cast<int>(rows), C,
+                                            tickets, losses, stream, true);
+        if (st != DB_OK) return st;
+    }
     // 3. one gradient per worker: G_w = X_w^T E_w, reduction over that worker's rows only
     {
         tc::GemmArgs a{};
@@ -623,7 +653,7 @@ extern "C" db_status db_worker_grad_grouped(const float* X, const int32_t* y, co
             gr.out[w] = G[w];
             gr.K[w] = offsets[w + 1] - offsets[w];
         }
-        const db_status st = launch_tc_gemm(a, 64, stream, &gr, K);
+        const db_status st = launch_tc_gemm(a, 64, stream, &gr, K, true);
         if (st != DB_OK) return st;
     }
     return DB_OK;
