@@ -249,51 +249,54 @@ __device__ __forceinline__ void tile_load(TileRegs<ROWS>& t, const float* __rest
     }
 }
 
-// Phase 2: split into TF32 halves and store into the swizzled hi / lo tiles.
+// Phase 2: split into TF32 halves and store into the swizzled hi / lo tiles.  `lo_delta` is the byte
+// distance from the hi tile to the lo tile.  A thread's elements sit at a fixed swizzled offset plus a
+// compile-time multiple of whole 8-row groups, so every store is [register + immediate].
 template <int ROWS, int MODE>
-__device__ __forceinline__ void tile_store(const TileRegs<ROWS>& t, unsigned char* hi_tile, unsigned char* lo_tile,
-                                           int tid) {
+__device__ __forceinline__ void tile_store(const TileRegs<ROWS>& t, unsigned char* hi_tile, int lo_delta, int tid) {
     const int warp = tid >> 5, lane = tid & 31;
     if (MODE == kLoadKVec) {
-        const int kk = (tid & 7) * 4;
+        // rows (tid >> 3) + 32 i: the row's position in its 8-row group never changes
+        unsigned char* base = hi_tile + swz(tid >> 3, (tid & 7) * 4);
 #pragma unroll
         for (int i = 0; i < ROWS / (kLoaderThreads / 8); ++i) {
-            const int r = (tid >> 3) + i * (kLoaderThreads / 8);
             float4 h, l;
             split_tf32(t.v[4 * i + 0], h.x, l.x);
             split_tf32(t.v[4 * i + 1], h.y, l.y);
             split_tf32(t.v[4 * i + 2], h.z, l.z);
             split_tf32(t.v[4 * i + 3], h.w, l.w);
-            const uint32_t off = swz(r, kk);
-            *reinterpret_cast<float4*>(hi_tile + off) = h;
-            *reinterpret_cast<float4*>(lo_tile + off) = l;
+            unsigned char* dst = base + i * (kLoaderThreads / 8) * 128;
+            *reinterpret_cast<float4*>(dst) = h;
+            *reinterpret_cast<float4*>(dst + lo_delta) = l;
         }
     } else if (MODE == kLoadRowVec) {
-        const int kl = lane >> 1, rsub = (lane & 1) * 4;
+        // step = warp + 8 i: k half (warp & 1) and the row's position in its group are fixed per thread
+        const int kk = (warp & 1) * 16 + (lane >> 1), r0 = (warp >> 1) * 8 + (lane & 1) * 4;
+        unsigned char* base[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) base[j] = hi_tile + swz(r0 + j, kk);
 #pragma unroll
         for (int i = 0; i < ROWS / (4 * kLoaderWarps); ++i) {
-            const int step = warp + i * kLoaderWarps;
-            const int r = (step >> 1) * 8 + rsub, kk = (step & 1) * 16 + kl;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 float h, l;
                 split_tf32(t.v[4 * i + j], h, l);
-                const uint32_t off = swz(r + j, kk);
-                *reinterpret_cast<float*>(hi_tile + off) = h;
-                *reinterpret_cast<float*>(lo_tile + off) = l;
+                unsigned char* dst = base[j] + i * (kLoaderWarps / 2) * 8 * 128;
+                *reinterpret_cast<float*>(dst) = h;
+                *reinterpret_cast<float*>(dst + lo_delta) = l;
             }
         }
     } else {
-        const int rl = lane & 7, kl = lane >> 3;
+        // patch = warp + 8 i: k group (warp & 7 ... ) fixed, row group advances by one per step
+        const int rl = lane & 7, kk = (warp & 7) * 4 + (lane >> 3);
+        unsigned char* base = hi_tile + swz(rl, kk);
 #pragma unroll
         for (int i = 0; i < ROWS / kLoaderWarps; ++i) {
-            const int pidx = warp + i * kLoaderWarps;
-            const int r = (pidx >> 3) * 8 + rl, kk = (pidx & 7) * 4 + kl;
             float h, l;
             split_tf32(t.v[i], h, l);
-            const uint32_t off = swz(r, kk);
-            *reinterpret_cast<float*>(hi_tile + off) = h;
-            *reinterpret_cast<float*>(lo_tile + off) = l;
+            unsigned char* dst = base + i * 8 * 128;       // (warp + 8 i) >> 3 = i row groups of 8
+            *reinterpret_cast<float*>(dst) = h;
+            *reinterpret_cast<float*>(dst + lo_delta) = l;
         }
     }
 }
@@ -318,6 +321,7 @@ __device__ __forceinline__ void tf32x3_gemm_body(const GemmArgs& g, const int sp
     constexpr int kStagePitch = N_TILE + 4;   // floats per row of the output staging tile (16-byte rows, no bank conflicts)
     static_assert(kTileM * kStagePitch * 4 <= kStages * L::kStage, "output staging fits in the operand stages");
     static_assert(N_TILE == 32 || N_TILE == 64 || N_TILE == 128, "accumulator columns: power of two >= 32");
+    static_assert(kLoaderWarps == 8, "the tile_load / tile_store lane maps assume eight loader warps");
     extern __shared__ unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kStages];
     __shared__ __align__(8) uint64_t empty_bar[kStages];
@@ -382,8 +386,8 @@ __device__ __forceinline__ void tf32x3_gemm_body(const GemmArgs& g, const int sp
                 alive = mbar_wait(&empty_bar[s], ((kb / kStages) - 1) & 1, &abort_flag, g.status, 1);
             if (!alive) break;
             unsigned char* st = tiles + s * L::kStage;
-            tile_store<kTileM, MODE_A>(ra, st, st + L::kATile, tid);
-            tile_store<N_TILE, MODE_B>(rb, st + 2 * L::kATile, st + 2 * L::kATile + L::kBTile, tid);
+            tile_store<kTileM, MODE_A>(ra, st, L::kATile, tid);
+            tile_store<N_TILE, MODE_B>(rb, st + 2 * L::kATile, L::kBTile, tid);
             fence_proxy_async_smem();   // make the generic-proxy stores visible to the tensor core
             mbar_arrive(&full_bar[s]);
             ra = ra_next;
