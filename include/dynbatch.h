@@ -125,6 +125,45 @@ db_status db_aggregate_adam_ex(const void* const* grads, db_dtype grad_dtype,
                                size_t workspace_bytes, void* cuda_stream);
 
 /* ------------------------------------------------------------------------
+ * The momentum step over a list of tensors        (Section 3.1, Eq. 2-3)
+ *
+ * For models whose T parameter tensors (and their gradients and momentum
+ * buffers) are separate allocations rather than one arena.  A plan is built
+ * once for a fixed set of tensors; each step is then one launch over all of
+ * them, with results bit-identical to db_aggregate_update_ex applied tensor by
+ * tensor (the squared norm is the sum over all tensors).
+ *
+ *   grads        host array of K*T device pointers, grads[k*T + t] = worker k's
+ *                gradient of tensor t (sizes[t] elements of grad_dtype)
+ *   sizes        host, T element counts >= 0
+ *   params, momentum   host arrays of T device pointers (fp32, sizes[t] each)
+ *   device_table device scratch of >= db_multi_plan_device_bytes(...) bytes,
+ *                256-byte aligned; the plan keeps its tensor descriptors, the
+ *                pointer table, one record per CTA and the norm's partial sums
+ *                there until it is destroyed.  Must outlive the plan.
+ *   cuda_stream  (create) the tables are uploaded on it and the call waits for
+ *                the upload; (step) the launch stream
+ * A tensor whose buffers are all 16-byte aligned takes 128-bit accesses,
+ * otherwise element-wise ones.  b[k] == 0: worker k's buffers are not read.
+ * The buffers of different tensors must not overlap; steps on one plan must not
+ * overlap on the device.
+ * ------------------------------------------------------------------------ */
+typedef struct db_multi_plan db_multi_plan;
+
+size_t db_multi_plan_device_bytes(int32_t K, db_dtype grad_dtype,
+                                  const int64_t* sizes, int32_t T);
+db_status db_multi_plan_create(db_multi_plan** out, const void* const* grads,
+                               db_dtype grad_dtype, int32_t K,
+                               const int64_t* sizes, int32_t T,
+                               float* const* params, float* const* momentum,
+                               void* device_table, size_t device_table_bytes,
+                               void* cuda_stream);
+db_status db_aggregate_update_multi(db_multi_plan* plan, const int32_t* b,
+                                    float lr, float mu, double* grad_sqnorm,
+                                    void* cuda_stream);
+db_status db_multi_plan_destroy(db_multi_plan* plan);
+
+/* ------------------------------------------------------------------------
  * The same step for callers that cannot provide scratch memory
  * (the paper has no counterpart; this is a packaging variant of the call above)
  *

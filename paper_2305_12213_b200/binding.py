@@ -42,6 +42,11 @@ _SIGNATURES = {
     "db_aggregate_adam_ex": (c_int32, [c_void_p, c_int32, c_void_p, c_int32, c_int64, c_void_p, c_void_p, c_void_p,
                                        c_float, c_float, c_float, c_float, c_int64, c_void_p, c_void_p, c_size_t,
                                        c_void_p]),
+    "db_multi_plan_device_bytes": (c_size_t, [c_int32, c_int32, c_void_p, c_int32]),
+    "db_multi_plan_create": (c_int32, [c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_int32, c_void_p, c_void_p,
+                                       c_void_p, c_size_t, c_void_p]),
+    "db_aggregate_update_multi": (c_int32, [c_void_p, c_void_p, c_float, c_float, c_void_p, c_void_p]),
+    "db_multi_plan_destroy": (c_int32, [c_void_p]),
     "db_aggregate_update_static": (c_int32, [c_void_p, c_int32, c_void_p, c_int32, c_int64, c_void_p,
                                              c_void_p, c_float, c_float, c_void_p, c_void_p]),
     "db_host_pipeline_create": (c_int32, [c_void_p]),
@@ -374,6 +379,56 @@ class Controller:
     def close(self) -> None:
         if self._h:
             lib().db_controller_destroy(self._h)
+            self._h = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class MultiTensorPlan:
+    """db_multi_plan: the momentum step over a fixed list of separately allocated tensors.
+
+    grads[k][t] is worker k's gradient of tensor t; params[t], momentum[t] its fp32 state.
+    """
+
+    def __init__(self, grads: Sequence[Sequence[torch.Tensor]], params: Sequence[torch.Tensor],
+                 momentum: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None):
+        K, T = len(grads), len(params)
+        gdt = grads[0][0].dtype
+        self.K = K
+        sizes = (c_int64 * T)(*[int(p.numel()) for p in params])
+        gtab = (c_void_p * (K * T))(*[_dev_ptr(grads[k][t], gdt, "grads[k][t]") for k in range(K) for t in range(T)])
+        ptab = (c_void_p * T)(*[_dev_ptr(p, torch.float32, "params[t]") for p in params])
+        vtab = (c_void_p * T)(*[_dev_ptr(v, torch.float32, "momentum[t]") for v in momentum])
+        for k in range(K):
+            for t in range(T):
+                if grads[k][t].numel() != params[t].numel():
+                    raise ValueError("gradient and parameter sizes differ")
+        code = _dtype_code(gdt)
+        nbytes = int(lib().db_multi_plan_device_bytes(K, code, ctypes.cast(sizes, c_void_p), T))
+        self.table = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=params[0].device)
+        self._keep = (list(params), list(momentum), [list(g) for g in grads])   # the plan stores raw pointers
+        self._h = c_void_p()
+        _check(lib().db_multi_plan_create(ctypes.byref(self._h), ctypes.cast(gtab, c_void_p), code, K,
+                                          ctypes.cast(sizes, c_void_p), T, ctypes.cast(ptab, c_void_p),
+                                          ctypes.cast(vtab, c_void_p), self.table.data_ptr(), self.table.numel(),
+                                          _stream_ptr(stream)))
+
+    def step(self, b: Sequence[int], lr: float, mu: float, grad_sqnorm: Optional[torch.Tensor] = None,
+             stream: Optional[torch.cuda.Stream] = None) -> None:
+        """db_aggregate_update_multi: one launch over every tensor of the plan."""
+        if len(b) != self.K:
+            raise ValueError("len(b) != K")
+        _check(lib().db_aggregate_update_multi(self._h, ctypes.cast(_i32_array(b), c_void_p), float(lr), float(mu),
+                                               _dev_ptr(grad_sqnorm, torch.float64, "grad_sqnorm"),
+                                               _stream_ptr(stream)))
+
+    def close(self) -> None:
+        if self._h:
+            lib().db_multi_plan_destroy(self._h)
             self._h = c_void_p()
 
     def __del__(self):

@@ -1,0 +1,90 @@
+// Device helpers shared by the aggregation kernels: gradient vector access for fp32 / bf16 storage,
+// the ordered block reduction and the "last CTA folds the partials" epilogue of the gradient norm.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace dynbatch {
+namespace agg {
+
+constexpr int kBlock = 256;
+constexpr int kChunk = 8;        // gradient slices loaded per round when K is not a compile-time constant
+
+// Raw 16-byte gradient vector and its widening to fp32 lanes.
+template <typename GT> struct GradVec;
+
+template <> struct GradVec<float> {
+    static constexpr int kLanes = 4;
+    using Raw = float4;
+    static __device__ __forceinline__ Raw load(const void* base, long long head, long long vi) {
+        return __ldcs(reinterpret_cast<const float4*>(static_cast<const float*>(base) + head) + vi);
+    }
+    static __device__ __forceinline__ void widen(const Raw& r, float (&x)[4]) {
+        x[0] = r.x; x[1] = r.y; x[2] = r.z; x[3] = r.w;
+    }
+    static __device__ __forceinline__ float scalar(const void* base, long long j) {
+        return __ldcs(static_cast<const float*>(base) + j);
+    }
+};
+
+template <> struct GradVec<__nv_bfloat16> {
+    static constexpr int kLanes = 8;
+    using Raw = uint4;
+    static __device__ __forceinline__ Raw load(const void* base, long long head, long long vi) {
+        return __ldcs(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(base) + head) + vi);
+    }
+    // bf16 is the high half of a binary32: widening is a shift, exact.
+    static __device__ __forceinline__ void widen(const Raw& r, float (&x)[8]) {
+        x[0] = __uint_as_float(r.x << 16); x[1] = __uint_as_float(r.x & 0xffff0000u);
+        x[2] = __uint_as_float(r.y << 16); x[3] = __uint_as_float(r.y & 0xffff0000u);
+        x[4] = __uint_as_float(r.z << 16); x[5] = __uint_as_float(r.z & 0xffff0000u);
+        x[6] = __uint_as_float(r.w << 16); x[7] = __uint_as_float(r.w & 0xffff0000u);
+    }
+    static __device__ __forceinline__ float scalar(const void* base, long long j) {
+        const uint16_t h = __ldcs(static_cast<const uint16_t*>(base) + j);
+        return __uint_as_float(static_cast<uint32_t>(h) << 16);
+    }
+};
+
+// Block-wide sum of doubles in a fixed order (xor tree in the warp, warps in order).
+__device__ __forceinline__ double block_sum(double x, double* smem) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();
+    if (lane == 0) smem[warp] = x;
+    __syncthreads();
+    double s = 0.0;
+    if (threadIdx.x == 0) {
+        for (int w = 0; w < kBlock / 32; ++w) s += smem[w];
+    }
+    return s;  // valid in thread 0
+}
+
+// Publishes this CTA's partial; the last CTA to arrive folds all partials in
+// index order.  No CTA ever waits on another: arrival order is taken from an
+// atomic ticket (zero at launch), so the kernel cannot spin.
+__device__ __forceinline__ void finish_norm(double* partials, unsigned int* ticket, double* sq_out, double sq) {
+    __shared__ double smem[kBlock / 32];
+    __shared__ bool is_last;
+    const double s = block_sum(sq, smem);
+    if (threadIdx.x == 0) {
+        partials[blockIdx.x] = s;
+        __threadfence();
+        const unsigned int t = atomicAdd(ticket, 1u);
+        is_last = (t == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    double acc = 0.0;
+    for (unsigned int i = threadIdx.x; i < gridDim.x; i += kBlock)
+        acc += __ldcg(partials + i);
+    const double total = block_sum(acc, smem);
+    if (threadIdx.x == 0) *sq_out = total;
+}
+
+}  // namespace agg
+}  // namespace dynbatch

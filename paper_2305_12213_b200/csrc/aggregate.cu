@@ -17,13 +17,15 @@
 #include <cstdint>
 #include <cstdio>
 
+#include "agg_device.cuh"
 #include "common.h"
 
 namespace dynbatch {
 namespace {
 
-constexpr int kBlock = 256;
-constexpr int kChunk = 8;        // gradient slices loaded per round beyond that
+using agg::GradVec;
+using agg::kBlock;
+using agg::kChunk;
 
 struct AggArgs {
     const void* g[DB_MAX_K];  // active workers' gradient buffers
@@ -59,80 +61,6 @@ __device__ __forceinline__ void optimizer_step(const AggArgs& a, float g, float&
         const float denom = sqrtf(u * a.inv_c2) + a.eps;
         p = p - a.lr * (v * a.inv_c1) / denom;
     }
-}
-
-// Raw 16-byte gradient vector and its widening to fp32 lanes.
-template <typename GT> struct GradVec;
-
-template <> struct GradVec<float> {
-    static constexpr int kLanes = 4;
-    using Raw = float4;
-    static __device__ __forceinline__ Raw load(const void* base, long long head, long long vi) {
-        return __ldcs(reinterpret_cast<const float4*>(static_cast<const float*>(base) + head) + vi);
-    }
-    static __device__ __forceinline__ void widen(const Raw& r, float (&x)[4]) {
-        x[0] = r.x; x[1] = r.y; x[2] = r.z; x[3] = r.w;
-    }
-    static __device__ __forceinline__ float scalar(const void* base, long long j) {
-        return __ldcs(static_cast<const float*>(base) + j);
-    }
-};
-
-template <> struct GradVec<__nv_bfloat16> {
-    static constexpr int kLanes = 8;
-    using Raw = uint4;
-    static __device__ __forceinline__ Raw load(const void* base, long long head, long long vi) {
-        return __ldcs(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(base) + head) + vi);
-    }
-    // bf16 is the high half of a binary32: widening is a shift, exact.
-    static __device__ __forceinline__ void widen(const Raw& r, float (&x)[8]) {
-        x[0] = __uint_as_float(r.x << 16); x[1] = __uint_as_float(r.x & 0xffff0000u);
-        x[2] = __uint_as_float(r.y << 16); x[3] = __uint_as_float(r.y & 0xffff0000u);
-        x[4] = __uint_as_float(r.z << 16); x[5] = __uint_as_float(r.z & 0xffff0000u);
-        x[6] = __uint_as_float(r.w << 16); x[7] = __uint_as_float(r.w & 0xffff0000u);
-    }
-    static __device__ __forceinline__ float scalar(const void* base, long long j) {
-        const uint16_t h = __ldcs(static_cast<const uint16_t*>(base) + j);
-        return __uint_as_float(static_cast<uint32_t>(h) << 16);
-    }
-};
-
-// Block-wide sum of doubles in a fixed order (xor tree in the warp, warps in order).
-__device__ __forceinline__ double block_sum(double x, double* smem) {
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    __syncthreads();
-    if (lane == 0) smem[warp] = x;
-    __syncthreads();
-    double s = 0.0;
-    if (threadIdx.x == 0) {
-        for (int w = 0; w < kBlock / 32; ++w) s += smem[w];
-    }
-    return s;  // valid in thread 0
-}
-
-// Publishes this CTA's partial; the last CTA to arrive folds all partials in
-// index order.  No CTA ever waits on another: arrival order is taken from an
-// atomic ticket, so the kernel cannot spin.
-__device__ __forceinline__ void finish_norm(const AggArgs& a, double sq) {
-    __shared__ double smem[kBlock / 32];
-    __shared__ bool is_last;
-    const double s = block_sum(sq, smem);
-    if (threadIdx.x == 0) {
-        a.partials[blockIdx.x] = s;
-        __threadfence();
-        const unsigned int t = atomicAdd(a.ticket, 1u);
-        is_last = (t == gridDim.x - 1);
-    }
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-    double acc = 0.0;
-    for (unsigned int i = threadIdx.x; i < gridDim.x; i += kBlock)
-        acc += __ldcg(a.partials + i);
-    const double total = block_sum(acc, smem);
-    if (threadIdx.x == 0) *a.sq_out = total;
 }
 
 // One element, any alignment: the same FMA chain as the vector body.
@@ -267,7 +195,7 @@ agg_vec_kernel(const __grid_constant__ AggArgs a) {
         if (threadIdx.x < a.head) update_scalar<GT, NORM, OPT>(a, K, threadIdx.x, sq);
         if (tail0 + threadIdx.x < a.n) update_scalar<GT, NORM, OPT>(a, K, tail0 + threadIdx.x, sq);
     }
-    if (NORM) finish_norm(a, sq);
+    if (NORM) agg::finish_norm(a.partials, a.ticket, a.sq_out, sq);
 }
 
 // Element-wise kernel for buffers whose 16-byte boundaries do not line up.
@@ -278,7 +206,7 @@ agg_scalar_kernel(const __grid_constant__ AggArgs a) {
     const long long step = static_cast<long long>(gridDim.x) * kBlock;
     for (long long j = static_cast<long long>(blockIdx.x) * kBlock + threadIdx.x; j < a.n; j += step)
         update_scalar<GT, NORM, OPT>(a, a.K, j, sq);
-    if (NORM) finish_norm(a, sq);
+    if (NORM) agg::finish_norm(a.partials, a.ticket, a.sq_out, sq);
 }
 
 // ---------------------------------------------------------------------------
