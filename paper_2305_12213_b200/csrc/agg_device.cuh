@@ -9,7 +9,7 @@
 namespace dynbatch {
 namespace agg {
 
-constexpr int kBlock = 256;
+constexpr int kBlock = 256;      // default CTA size; kernels may run with fewer threads (a multiple of 32)
 constexpr int kChunk = 8;        // gradient slices loaded per round when K is not a compile-time constant
 
 // Raw 16-byte gradient vector and its widening to fp32 lanes.
@@ -58,7 +58,7 @@ __device__ __forceinline__ double block_sum(double x, double* smem) {
     __syncthreads();
     double s = 0.0;
     if (threadIdx.x == 0) {
-        for (int w = 0; w < kBlock / 32; ++w) s += smem[w];
+        for (int w = 0; w < static_cast<int>(blockDim.x) / 32; ++w) s += smem[w];
     }
     return s;  // valid in thread 0
 }
@@ -80,7 +80,7 @@ __device__ __forceinline__ void finish_norm(double* partials, unsigned int* tick
     if (!is_last) return;
     __threadfence();
     double acc = 0.0;
-    for (unsigned int i = threadIdx.x; i < gridDim.x; i += kBlock)
+    for (unsigned int i = threadIdx.x; i < gridDim.x; i += blockDim.x)
         acc += __ldcg(partials + i);
     const double total = block_sum(acc, smem);
     if (threadIdx.x == 0) *sq_out = total;

@@ -102,9 +102,9 @@ __device__ __forceinline__ void apply_update(const AggArgs& a, long long vi, con
 }
 
 // KT > 0: exactly KT workers, fully unrolled.  KT == 0: a.K workers, kChunk at a time.
-// A CTA handles TILES consecutive tiles of kBlock x UNROLL vectors.
-template <typename GT, int KT, int UNROLL, int TILES, bool NORM, int OPT>
-__global__ void __launch_bounds__(kBlock)
+// A CTA of BLOCK threads handles TILES consecutive tiles of BLOCK x UNROLL vectors.
+template <typename GT, int KT, int BLOCK, int UNROLL, int TILES, bool NORM, int OPT>
+__global__ void __launch_bounds__(BLOCK)
 agg_vec_kernel(const __grid_constant__ AggArgs a) {
     using GV = GradVec<GT>;
     using Raw = typename GV::Raw;
@@ -113,7 +113,7 @@ agg_vec_kernel(const __grid_constant__ AggArgs a) {
     const int K = KT > 0 ? KT : a.K;
     double sq = 0.0;
 
-    const long long tile = static_cast<long long>(kBlock) * UNROLL;
+    const long long tile = static_cast<long long>(BLOCK) * UNROLL;
 #pragma unroll 1
     for (int t = 0; t < TILES; ++t) {
         const long long base = (static_cast<long long>(blockIdx.x) * TILES + t) * tile;
@@ -124,7 +124,7 @@ agg_vec_kernel(const __grid_constant__ AggArgs a) {
         float g[UNROLL][kLanes];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-            vi[u] = base + u * kBlock + threadIdx.x;
+            vi[u] = base + u * BLOCK + threadIdx.x;
             ok[u] = vi[u] < a.nvec;
 #pragma unroll
             for (int l = 0; l < kLanes; ++l) g[u][l] = 0.0f;
@@ -217,25 +217,32 @@ constexpr size_t kTicketBytes = 256;  // ticket word, padded so the partials sta
 using KernelFn = void (*)(const AggArgs);
 
 template <typename GT, int KT, bool NORM, int OPT>
-KernelFn pick_unroll(int* vectors_per_cta) {
-    // Measured on B200 (with the norm): up to 8 workers, two vector positions per thread and one tile
-    // per CTA (2 (K + 2) independent 16-byte loads in flight per thread); 9 to 16 workers, one position
-    // per thread (registers) and two consecutive tiles per CTA, which amortises the norm epilogue;
-    // the chunked many-worker kernel one tile (more tiles per CTA cost it 30 %).
-    constexpr int kUnroll = (KT >= 1 && KT <= 8) ? 2 : 1;
+KernelFn pick_unroll(int* vectors_per_cta, int* block) {
+    // Launch shapes measured on B200 (with the norm), fp32 and bf16 gradients:
+    //   up to 8 workers   256 threads, two vector positions per thread, one tile per CTA
+    //                     (2 (K + 2) independent 16-byte loads in flight per thread);
+    //   9 to 16 workers   128 threads, two positions, two consecutive tiles per CTA: the smaller CTA
+    //                     keeps two resident per SM despite ~40 loads per thread, and the second tile
+    //                     amortises the norm epilogue (bf16, K = 16: 6.9 TB/s against 6.3-6.6 for
+    //                     every 256-thread shape);
+    //   more workers      the chunked kernel, 256 threads, one position, one tile (more tiles per CTA
+    //                     cost it 30 %).
+    constexpr int kThreads = (KT >= 9) ? 128 : kBlock;
+    constexpr int kUnroll = (KT >= 1) ? 2 : 1;
     constexpr int kTiles = (KT >= 9) ? 2 : 1;
-    *vectors_per_cta = kBlock * kUnroll * kTiles;
-    return agg_vec_kernel<GT, KT, kUnroll, kTiles, NORM, OPT>;
+    *vectors_per_cta = kThreads * kUnroll * kTiles;
+    *block = kThreads;
+    return agg_vec_kernel<GT, KT, kThreads, kUnroll, kTiles, NORM, OPT>;
 }
 
 template <typename GT, bool NORM, int OPT>
-KernelFn pick_vec_kernel(int K, int* unroll_out) {
+KernelFn pick_vec_kernel(int K, int* unroll_out, int* block) {
     switch (K) {
-#define DB_CASE(n) case n: return pick_unroll<GT, n, NORM, OPT>(unroll_out);
+#define DB_CASE(n) case n: return pick_unroll<GT, n, NORM, OPT>(unroll_out, block);
         DB_CASE(1) DB_CASE(2) DB_CASE(3) DB_CASE(4) DB_CASE(5) DB_CASE(6) DB_CASE(7) DB_CASE(8)
         DB_CASE(9) DB_CASE(10) DB_CASE(11) DB_CASE(12) DB_CASE(13) DB_CASE(14) DB_CASE(15) DB_CASE(16)
 #undef DB_CASE
-        default: return pick_unroll<GT, 0, NORM, OPT>(unroll_out);
+        default: return pick_unroll<GT, 0, NORM, OPT>(unroll_out, block);
     }
 }
 
@@ -273,13 +280,14 @@ namespace dynbatch {
 namespace {
 
 template <int OPT>
-KernelFn pick_kernel(bool vector_ok, db_dtype dt, bool norm, int active, int* vectors_per_cta) {
+KernelFn pick_kernel(bool vector_ok, db_dtype dt, bool norm, int active, int* vectors_per_cta, int* block) {
+    *block = kBlock;
     if (vector_ok) {
         if (dt == DB_F32)
-            return norm ? pick_vec_kernel<float, true, OPT>(active, vectors_per_cta)
-                        : pick_vec_kernel<float, false, OPT>(active, vectors_per_cta);
-        return norm ? pick_vec_kernel<__nv_bfloat16, true, OPT>(active, vectors_per_cta)
-                    : pick_vec_kernel<__nv_bfloat16, false, OPT>(active, vectors_per_cta);
+            return norm ? pick_vec_kernel<float, true, OPT>(active, vectors_per_cta, block)
+                        : pick_vec_kernel<float, false, OPT>(active, vectors_per_cta, block);
+        return norm ? pick_vec_kernel<__nv_bfloat16, true, OPT>(active, vectors_per_cta, block)
+                    : pick_vec_kernel<__nv_bfloat16, false, OPT>(active, vectors_per_cta, block);
     }
     if (dt == DB_F32) return norm ? agg_scalar_kernel<float, true, OPT> : agg_scalar_kernel<float, false, OPT>;
     return norm ? agg_scalar_kernel<__nv_bfloat16, true, OPT> : agg_scalar_kernel<__nv_bfloat16, false, OPT>;
@@ -357,9 +365,10 @@ db_status aggregate_launch(AggArgs a, int opt, const void* const* grads, db_dtyp
     a.head = head;
     a.nvec = (N - head) / lanes;
 
-    int vectors_per_cta = kBlock;
-    const KernelFn fn = opt == kAdam ? pick_kernel<kAdam>(vector_ok, grad_dtype, norm, active, &vectors_per_cta)
-                                     : pick_kernel<kMomentum>(vector_ok, grad_dtype, norm, active, &vectors_per_cta);
+    int vectors_per_cta = kBlock, block = kBlock;
+    const KernelFn fn = opt == kAdam
+                            ? pick_kernel<kAdam>(vector_ok, grad_dtype, norm, active, &vectors_per_cta, &block)
+                            : pick_kernel<kMomentum>(vector_ok, grad_dtype, norm, active, &vectors_per_cta, &block);
     int grid;
     if (vector_ok) {
         const long long tiles = (a.nvec + vectors_per_cta - 1) / vectors_per_cta;
@@ -369,7 +378,7 @@ db_status aggregate_launch(AggArgs a, int opt, const void* const* grads, db_dtyp
         grid = scalar_grid(fn, N);
     }
     if (norm) DB_CUDA_TRY(cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), stream));
-    fn<<<grid, kBlock, 0, stream>>>(a);
+    fn<<<grid, block, 0, stream>>>(a);
     DB_CUDA_TRY(cudaGetLastError());
     return DB_OK;
 }
