@@ -13,6 +13,7 @@
 // The two contractions run on the tensor cores (tcgen05, three TF32 products per
 // fp32 product, see tc_gemm.cuh).  An fp32 FFMA version on shared-memory tiles is
 // kept as the accuracy reference and for very large b_i.
+#include <algorithm>
 #include <cstdint>
 
 #include "common.h"
@@ -647,11 +648,18 @@ extern "C" db_status db_worker_grad_grouped(const float* X, const int32_t* y, co
         a.o_m = C; a.o_n = 1; a.o_split = 0;
         a.M = D; a.N = C; a.status = status;
         tc::GroupArgs gr{};
-        for (int w = 0; w < K; ++w) {
-            gr.A[w] = X + static_cast<long long>(offsets[w]) * D;
-            gr.B[w] = E + static_cast<long long>(offsets[w]) * C;
-            gr.out[w] = G[w];
-            gr.K[w] = offsets[w + 1] - offsets[w];
+        // largest batches first: their CTAs run longest and should not form the tail of the grid
+        int order[DB_MAX_K];
+        for (int w = 0; w < K; ++w) order[w] = w;
+        std::stable_sort(order, order + K, [&](int u, int v) {
+            return offsets[u + 1] - offsets[u] > offsets[v + 1] - offsets[v];
+        });
+        for (int z = 0; z < K; ++z) {
+            const int w = order[z];
+            gr.A[z] = X + static_cast<long long>(offsets[w]) * D;
+            gr.B[z] = E + static_cast<long long>(offsets[w]) * C;
+            gr.out[z] = G[w];
+            gr.K[z] = offsets[w + 1] - offsets[w];
         }
         const db_status st = launch_tc_gemm(a, 64, stream, &gr, K, true);
         if (st != DB_OK) return st;
