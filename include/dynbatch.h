@@ -185,13 +185,13 @@ db_status db_multi_plan_destroy(db_multi_plan* plan);
  *     (once per device, with that device current).  Make that first call
  *     outside any stream capture.
  *   - All calls on a device share the one array.  It keeps the previous
- *     call's contents; the part that must start at zero (the CTA arrival
- *     counter) is cleared on the stream ahead of every launch.  Two calls
+ *     call's contents; nothing in it has to start at zero, since every CTA
+ *     of a launch overwrites its own slot before the fold reads it.  Two calls
  *     whose kernels may run at the same time on one device (different
  *     streams, different threads) race on it and return a wrong norm:
  *     serialise them, or use db_aggregate_update_ex with separate workspaces.
  *   - The scratch holds one double per CTA, i.e. per 1024 parameters, so the
- *     built-in 1 MiB serves N up to 134,182,912 parameters when the norm is
+ *     built-in 1 MiB serves N up to 134,215,680 parameters when the norm is
  *     requested (any N without it).  Beyond that the call returns
  *     DB_ERR_UNSUPPORTED and enqueues nothing; db_last_cuda_error() then says
  *     how many bytes were needed.

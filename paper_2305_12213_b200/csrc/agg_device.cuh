@@ -1,5 +1,6 @@
 // Device helpers shared by the aggregation kernels: gradient vector access for fp32 / bf16 storage,
-// the ordered block reduction and the "last CTA folds the partials" epilogue of the gradient norm.
+// the ordered block reduction, and the gradient norm's epilogue (one partial per CTA, folded by a
+// one-CTA kernel that is launched behind the aggregation kernel).
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -63,27 +64,48 @@ __device__ __forceinline__ double block_sum(double x, double* smem) {
     return s;  // valid in thread 0
 }
 
-// Publishes this CTA's partial; the last CTA to arrive folds all partials in
-// index order.  No CTA ever waits on another: arrival order is taken from an
-// atomic ticket (zero at launch), so the kernel cannot spin.
-__device__ __forceinline__ void finish_norm(double* partials, unsigned int* ticket, double* sq_out, double sq) {
+// Programmatic dependent launch (no-ops for kernels launched without the attribute): let the next
+// kernel in the stream be scheduled while this one runs / wait until the previous kernel has
+// completed and its writes are visible.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Gradient norm, step 1: every CTA of an aggregation kernel leaves the sum of its squared
+// aggregated gradients in partials[blockIdx.x].
+__device__ __forceinline__ void store_norm_partial(double* partials, double sq) {
     __shared__ double smem[kBlock / 32];
-    __shared__ bool is_last;
     const double s = block_sum(sq, smem);
-    if (threadIdx.x == 0) {
-        partials[blockIdx.x] = s;
-        __threadfence();
-        const unsigned int t = atomicAdd(ticket, 1u);
-        is_last = (t == gridDim.x - 1);
-    }
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
+    if (threadIdx.x == 0) partials[blockIdx.x] = s;
+}
+
+// Gradient norm, step 2: one CTA folds the n partials in index order.  Launched right behind the
+// aggregation kernel with programmatic stream serialization, so its launch latency is hidden; it
+// touches the partials only after griddepcontrol.wait.  No counter, nothing to initialise, nobody spins.
+static __global__ void __launch_bounds__(1024) norm_finalize_kernel(const double* __restrict__ partials, long long n,
+                                                             double* __restrict__ sq_out) {
+    __shared__ double smem[32];
+    griddep_wait();
     double acc = 0.0;
-    for (unsigned int i = threadIdx.x; i < gridDim.x; i += blockDim.x)
-        acc += __ldcg(partials + i);
+    for (long long i = threadIdx.x; i < n; i += blockDim.x) acc += __ldcg(partials + i);
     const double total = block_sum(acc, smem);
     if (threadIdx.x == 0) *sq_out = total;
+}
+
+// Enqueues norm_finalize_kernel behind the kernel just launched on `stream`; `overlap` lets it be scheduled
+// while that kernel still runs.
+static inline cudaError_t launch_norm_finalize(const double* partials, long long n, double* sq_out, cudaStream_t stream,
+                                               bool overlap) {
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1]{};
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3(n > 8192 ? 1024 : 256);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;   // without the attribute the kernel simply runs after its predecessor
+    return cudaLaunchKernelEx(&cfg, norm_finalize_kernel, partials, n, sq_out);
 }
 
 }  // namespace agg

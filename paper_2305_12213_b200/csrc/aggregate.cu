@@ -34,7 +34,6 @@ struct AggArgs {
     float* v;                 // momentum (heavy ball) or first moment (Adam)
     float* u;                 // second moment (Adam only)
     double* partials;         // one per CTA (norm only)
-    unsigned int* ticket;     // CTA arrival counter, zero at launch (norm only)
     double* sq_out;
     long long n;              // elements
     long long head;           // leading elements before the first 16-byte boundary
@@ -112,6 +111,7 @@ agg_vec_kernel(const __grid_constant__ AggArgs a) {
     constexpr int kQuads = kLanes / 4;
     const int K = KT > 0 ? KT : a.K;
     double sq = 0.0;
+    if (NORM) agg::griddep_launch_dependents();   // the norm's finalize kernel may be scheduled already
 
     const long long tile = static_cast<long long>(BLOCK) * UNROLL;
 #pragma unroll 1
@@ -195,7 +195,7 @@ agg_vec_kernel(const __grid_constant__ AggArgs a) {
         if (threadIdx.x < a.head) update_scalar<GT, NORM, OPT>(a, K, threadIdx.x, sq);
         if (tail0 + threadIdx.x < a.n) update_scalar<GT, NORM, OPT>(a, K, tail0 + threadIdx.x, sq);
     }
-    if (NORM) agg::finish_norm(a.partials, a.ticket, a.sq_out, sq);
+    if (NORM) agg::store_norm_partial(a.partials, sq);
 }
 
 // Element-wise kernel for buffers whose 16-byte boundaries do not line up.
@@ -203,17 +203,16 @@ template <typename GT, bool NORM, int OPT>
 __global__ void __launch_bounds__(kBlock)
 agg_scalar_kernel(const __grid_constant__ AggArgs a) {
     double sq = 0.0;
+    if (NORM) agg::griddep_launch_dependents();
     const long long step = static_cast<long long>(gridDim.x) * kBlock;
     for (long long j = static_cast<long long>(blockIdx.x) * kBlock + threadIdx.x; j < a.n; j += step)
         update_scalar<GT, NORM, OPT>(a, a.K, j, sq);
-    if (NORM) agg::finish_norm(a.partials, a.ticket, a.sq_out, sq);
+    if (NORM) agg::store_norm_partial(a.partials, sq);
 }
 
 // ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
-constexpr size_t kTicketBytes = 256;  // ticket word, padded so the partials stay aligned
-
 using KernelFn = void (*)(const AggArgs);
 
 template <typename GT, int KT, bool NORM, int OPT>
@@ -272,8 +271,8 @@ int scalar_grid(KernelFn fn, long long n) {
 
 extern "C" size_t db_aggregate_workspace_bytes(int32_t K, int64_t N) {
     (void)K;
-    // ticket + one double per CTA
-    return dynbatch::kTicketBytes + sizeof(double) * static_cast<size_t>(dynbatch::cta_bound(N < 0 ? 0 : N));
+    // one double per CTA
+    return sizeof(double) * static_cast<size_t>(dynbatch::cta_bound(N < 0 ? 0 : N));
 }
 
 namespace dynbatch {
@@ -297,7 +296,8 @@ KernelFn pick_kernel(bool vector_ok, db_dtype dt, bool norm, int active, int* ve
 // `a` arrives with the optimizer's scalars set; `second` is Adam's second-moment buffer (else NULL).
 db_status aggregate_launch(AggArgs a, int opt, const void* const* grads, db_dtype grad_dtype, const int32_t* b,
                            int32_t K, int64_t N, float* params, float* first, float* second,
-                           double* grad_sqnorm, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+                           double* grad_sqnorm, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                           double* chunk_partials = nullptr, long long* chunk_ctas = nullptr) {
     if (!grads || !b) return DB_ERR_NULL;
     if (K < 1 || K > DB_MAX_K || N < 0) return DB_ERR_ARG;
     if (grad_dtype != DB_F32 && grad_dtype != DB_BF16) return DB_ERR_UNSUPPORTED;
@@ -336,14 +336,16 @@ db_status aggregate_launch(AggArgs a, int opt, const void* const* grads, db_dtyp
     a.u = second;
     a.n = N;
 
-    const bool norm = grad_sqnorm != nullptr;
+    // chunk mode (the host pipeline): only the partial sums are produced, at a place the caller chose
+    const bool norm = grad_sqnorm != nullptr || chunk_partials != nullptr;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (norm) {
+    if (chunk_partials) {
+        a.partials = chunk_partials;
+    } else if (norm) {
         if (!workspace) return DB_ERR_NULL;
         if (reinterpret_cast<uintptr_t>(workspace) % 16 || workspace_bytes < db_aggregate_workspace_bytes(K, N))
             return DB_ERR_ARG;
-        a.ticket = static_cast<unsigned int*>(workspace);
-        a.partials = reinterpret_cast<double*>(static_cast<char*>(workspace) + kTicketBytes);
+        a.partials = static_cast<double*>(workspace);
         a.sq_out = grad_sqnorm;
     }
 
@@ -377,13 +379,33 @@ db_status aggregate_launch(AggArgs a, int opt, const void* const* grads, db_dtyp
     } else {
         grid = scalar_grid(fn, N);
     }
-    if (norm) DB_CUDA_TRY(cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), stream));
     fn<<<grid, block, 0, stream>>>(a);
     DB_CUDA_TRY(cudaGetLastError());
+    if (chunk_ctas) *chunk_ctas = grid;
+    if (norm && !chunk_partials) DB_CUDA_TRY(agg::launch_norm_finalize(a.partials, grid, a.sq_out, stream, true));
     return DB_OK;
 }
 
 }  // namespace
+
+long long aggregate_cta_bound(int64_t N) { return cta_bound(N < 0 ? 0 : N); }
+
+db_status aggregate_chunk(const void* const* grads, db_dtype grad_dtype, const int32_t* b, int32_t K, int64_t N,
+                          float* params, float* momentum, float lr, float mu, double* partials, long long* ctas,
+                          void* cuda_stream) {
+    if (ctas) *ctas = 0;
+    AggArgs a{};
+    a.lr = lr;
+    a.mu = mu;
+    return aggregate_launch(a, kMomentum, grads, grad_dtype, b, K, N, params, momentum, nullptr, nullptr, nullptr, 0,
+                            cuda_stream, partials, ctas);
+}
+
+db_status finalize_norm(const double* partials, long long n, double* sq_out, cudaStream_t stream) {
+    DB_CUDA_TRY(agg::launch_norm_finalize(partials, n, sq_out, stream, false));
+    return DB_OK;
+}
+
 }  // namespace dynbatch
 
 extern "C" db_status db_aggregate_update_ex(const void* const* grads, db_dtype grad_dtype,
@@ -432,7 +454,7 @@ extern "C" db_status db_aggregate_update(const float* const* grads, const int32_
 namespace dynbatch {
 namespace {
 
-// Ticket + per-CTA partials of the norm.  Lives in every device's global memory
+// Per-CTA partials of the norm.  Lives in every device's global memory
 // for the life of the process.  In host code this name is only a handle for
 // cudaGetSymbolAddress: it is never passed to a kernel as a pointer.
 static __device__ __align__(256) unsigned char g_static_scratch[DB_STATIC_SCRATCH_BYTES];

@@ -37,7 +37,6 @@ struct MultiArgs {
     const void* const* gptr;   // gptr[t * K + k]
     float lambda[DB_MAX_K];    // 0 for a worker with an empty batch: its buffers are not read
     double* partials;
-    unsigned int* ticket;
     double* sq_out;
     float lr, mu;
     int K;
@@ -63,6 +62,7 @@ agg_multi_kernel(const __grid_constant__ MultiArgs a) {
     using Raw = typename GV::Raw;
     constexpr int kLanes = GV::kLanes;
     constexpr int kQuads = kLanes / 4;
+    if (NORM) agg::griddep_launch_dependents();
     const TileRecord rec = a.tiles[blockIdx.x];
     const TensorDesc d = a.desc[rec.tensor];
     const void* const* g = a.gptr + static_cast<long long>(rec.tensor) * a.K;
@@ -133,10 +133,8 @@ agg_multi_kernel(const __grid_constant__ MultiArgs a) {
             if (j < d.n && j < e0 + static_cast<long long>(kBlock) * kLanes) multi_scalar<GT, NORM>(a, d, g, j, sq);
         }
     }
-    if (NORM) agg::finish_norm(a.partials, a.ticket, a.sq_out, sq);
+    if (NORM) agg::store_norm_partial(a.partials, sq);
 }
-
-constexpr size_t kTicketBytes = 256;
 
 size_t round256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
@@ -160,7 +158,7 @@ bool plan_layout(int32_t K, int32_t T, const int64_t* sizes, db_dtype dt, PlanLa
     }
     if (tiles > 0x7fffffffLL) return false;
     L->total_tiles = tiles;
-    L->partials_off = kTicketBytes;
+    L->partials_off = 0;
     L->desc_off = L->partials_off + round256(sizeof(double) * static_cast<size_t>(tiles > 0 ? tiles : 1));
     L->gptr_off = L->desc_off + round256(sizeof(TensorDesc) * static_cast<size_t>(T));
     L->tiles_off = L->gptr_off + round256(sizeof(void*) * static_cast<size_t>(T) * K);
@@ -252,7 +250,6 @@ extern "C" db_status db_multi_plan_create(db_multi_plan** out, const void* const
     plan->args.desc = reinterpret_cast<const TensorDesc*>(base + L.desc_off);
     plan->args.gptr = reinterpret_cast<const void* const*>(base + L.gptr_off);
     plan->args.partials = reinterpret_cast<double*>(base + L.partials_off);
-    plan->args.ticket = reinterpret_cast<unsigned int*>(base);
     plan->args.K = K;
     *out = plan;
     return DB_OK;
@@ -281,8 +278,8 @@ extern "C" db_status db_aggregate_update_multi(db_multi_plan* plan, const int32_
     void (*fn)(const MultiArgs);
     if (plan->dtype == DB_F32) fn = norm ? agg_multi_kernel<float, true> : agg_multi_kernel<float, false>;
     else fn = norm ? agg_multi_kernel<__nv_bfloat16, true> : agg_multi_kernel<__nv_bfloat16, false>;
-    if (norm) DB_CUDA_TRY(cudaMemsetAsync(a.ticket, 0, sizeof(unsigned int), stream));
     fn<<<static_cast<unsigned int>(plan->total_tiles), kBlock, 0, stream>>>(a);
     DB_CUDA_TRY(cudaGetLastError());
+    if (norm) DB_CUDA_TRY(agg::launch_norm_finalize(a.partials, plan->total_tiles, a.sq_out, stream, true));
     return DB_OK;
 }

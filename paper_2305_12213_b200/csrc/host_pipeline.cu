@@ -25,14 +25,6 @@ namespace {
 constexpr int64_t kDefaultChunk = 1 << 21;  // elements per chunk
 constexpr int kSlots = 2;
 
-__global__ void sum_chunk_norms_kernel(const double* __restrict__ parts, int n, double* __restrict__ total) {
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        double s = 0.0;
-        for (int i = 0; i < n; ++i) s += parts[i];
-        *total = s;
-    }
-}
-
 size_t round256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
 int64_t chunk_or_default(int64_t chunk_elems) {
@@ -41,7 +33,7 @@ int64_t chunk_or_default(int64_t chunk_elems) {
 }
 
 struct StagingLayout {
-    size_t slot_bytes, slots_off, ws_off, ws_bytes, norms_off, total_off, end;
+    size_t slot_bytes, slots_off, partials_off, total_off, end;
 };
 
 StagingLayout layout(int32_t K, db_dtype dt, int64_t N, int64_t chunk) {
@@ -49,11 +41,11 @@ StagingLayout layout(int32_t K, db_dtype dt, int64_t N, int64_t chunk) {
     const size_t gsize = dt == DB_F32 ? 4 : 2;
     L.slot_bytes = round256(static_cast<size_t>(K) * chunk * gsize);
     L.slots_off = 0;
-    L.ws_off = L.slots_off + kSlots * L.slot_bytes;
-    L.ws_bytes = round256(db_aggregate_workspace_bytes(K, chunk));
-    L.norms_off = L.ws_off + L.ws_bytes;
+    // every CTA of every chunk leaves one partial sum of the squared norm; one kernel folds them at the end
+    L.partials_off = L.slots_off + kSlots * L.slot_bytes;
     const int64_t nchunks = N > 0 ? (N + chunk - 1) / chunk : 1;
-    L.total_off = L.norms_off + round256(sizeof(double) * static_cast<size_t>(nchunks));
+    L.total_off = L.partials_off +
+                  round256(sizeof(double) * static_cast<size_t>(nchunks * aggregate_cta_bound(chunk)));
     L.end = L.total_off + 256;
     return L;
 }
@@ -130,8 +122,8 @@ extern "C" db_status db_aggregate_update_host(db_host_pipeline* h, const void* c
     cudaStream_t compute = static_cast<cudaStream_t>(cuda_stream);
     const size_t gsize = grad_dtype == DB_F32 ? 4 : 2;
     char* base = static_cast<char*>(staging);
-    void* ws = base + L.ws_off;
-    double* norms = reinterpret_cast<double*>(base + L.norms_off);
+    double* partials = reinterpret_cast<double*>(base + L.partials_off);
+    long long n_partials = 0;
     double* total_norm = reinterpret_cast<double*>(base + L.total_off);
     const int64_t nchunks = (N + chunk - 1) / chunk;
 
@@ -160,10 +152,11 @@ extern "C" db_status db_aggregate_update_host(db_host_pipeline* h, const void* c
 
         // compute on the caller's stream
         DB_CUDA_TRY(cudaStreamWaitEvent(compute, h->loaded[s], 0));
-        const db_status st = db_aggregate_update_ex(slices, grad_dtype, b, K, len, params + off, momentum + off,
-                                                    lr, mu, host_sqnorm_out ? norms + c : nullptr,
-                                                    host_sqnorm_out ? ws : nullptr, L.ws_bytes, compute);
+        long long ctas = 0;
+        const db_status st = aggregate_chunk(slices, grad_dtype, b, K, len, params + off, momentum + off, lr, mu,
+                                             host_sqnorm_out ? partials + n_partials : nullptr, &ctas, compute);
         if (st != DB_OK) return st;
+        n_partials += ctas;
         DB_CUDA_TRY(cudaEventRecord(h->computed[s], compute));
 
         // copy-out of the updated parameters
@@ -174,8 +167,8 @@ extern "C" db_status db_aggregate_update_host(db_host_pipeline* h, const void* c
         }
     }
     if (host_sqnorm_out) {
-        sum_chunk_norms_kernel<<<1, 32, 0, compute>>>(norms, static_cast<int>(nchunks), total_norm);
-        DB_CUDA_TRY(cudaGetLastError());
+        const db_status st = finalize_norm(partials, n_partials, total_norm, compute);
+        if (st != DB_OK) return st;
         DB_CUDA_TRY(cudaMemcpyAsync(host_sqnorm_out, total_norm, sizeof(double), cudaMemcpyDeviceToHost, compute));
     }
     // the caller's stream completes only after the last parameter chunk has reached the host

@@ -3,8 +3,7 @@
 Some users of the library may not allocate device memory at all (a plug-in whose host owns the whole
 GPU heap, a loop where cudaMalloc's device-wide synchronisation is not acceptable).  For them the
 norm's scratch lives in a fixed array inside the library.  The result must be the one the workspace
-form gives -- also on a second call, when the shared array still holds the first call's partials
-and arrival counter.  This file sorts last so a failure here cannot hide another test's.
+form gives -- also on a second call, when the shared array still holds the first call's partials.  This file sorts last so a failure here cannot hide another test's.
 """
 import pytest
 import torch
