@@ -511,34 +511,11 @@ __device__ __forceinline__ void tf32x3_gemm_body(const GemmArgs& g, const int sp
     }
 }
 
-// One problem, blockIdx.z = split of the reduction.
+// blockIdx.z = split of the reduction.
 template <int N_TILE, int MODE_A, int MODE_B>
 __global__ void __launch_bounds__(kThreads)
 tf32x3_gemm_kernel(const __grid_constant__ GemmArgs g) {
     tf32x3_gemm_body<N_TILE, MODE_A, MODE_B>(g, blockIdx.z);
-}
-
-// Several problems that share every stride, M and N but have their own operands, output and
-// reduction length (the ragged per-worker gradients): blockIdx.z = problem, no split.
-struct GroupArgs {
-    const float* A[DB_MAX_K];
-    const float* B[DB_MAX_K];
-    float* out[DB_MAX_K];
-    int K[DB_MAX_K];
-};
-
-template <int N_TILE, int MODE_A, int MODE_B>
-__global__ void __launch_bounds__(kThreads)
-tf32x3_gemm_grouped_kernel(const __grid_constant__ GemmArgs shared, const __grid_constant__ GroupArgs groups) {
-    GemmArgs g = shared;
-    const int z = blockIdx.z;
-    g.A = groups.A[z];
-    g.B = groups.B[z];
-    g.out = groups.out[z];
-    g.K = groups.K[z];
-    g.k_per_split = (g.K + kBlockK - 1) / kBlockK * kBlockK;
-    if (g.k_per_split == 0) g.k_per_split = kBlockK;
-    tf32x3_gemm_body<N_TILE, MODE_A, MODE_B>(g, 0);
 }
 
 }  // namespace tc

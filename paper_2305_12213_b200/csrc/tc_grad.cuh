@@ -1,0 +1,261 @@
+// The ragged gradient contraction on the tensor cores, fed by TMA (sm_100a):
+//     G_w(d, c) = sum_{r in worker w} X(r, d) * E(r, c)          for every worker w in one launch
+// X ([rows, D]) and E ([rows, C]) are row-major with the reduction index r as the row, so both
+// operands are contiguous along their OUTPUT index.  tcgen05.mma reads such "MN-major" tiles
+// directly, which removes the transposition through registers that the general contraction in
+// tc_gemm.cuh has to do; what is left of the operand preparation, the split of every fp32 value
+// into two TF32 halves, is done once by the kernel that produces E (and copies X), not once per
+// output tile.  A CTA of this kernel therefore only
+//   - copies [32 rows x 32 columns] boxes of the four split arrays (X_hi, X_lo, E_hi, E_lo) into
+//     shared memory with cp.async.bulk.tensor (128-byte swizzle of 32-byte pieces, completion on an
+//     mbarrier),
+//   - issues three tcgen05.mma.kind::tf32 per 8 rows (lo*hi + hi*lo into one accumulator in tensor
+//     memory, hi*hi round-robin into up to seven others, see tc_gemm.cuh for why), and
+//   - drains the accumulators and writes its 128 x 64 tile of G.
+// In the split arrays every worker's rows start at a multiple of 8 and are padded with zero rows to
+// a multiple of 8, the reduction depth of one TF32 product.
+//
+// 192 threads: warp 0 (one lane) issues the TMA copies, warp 1 owns the tensor-memory allocation
+// and (one lane) issues the products, warps 2-5 are the epilogue.  Two shared-memory stages of
+// 48 KB, so two CTAs fit on an SM and one's epilogue overlaps the other's loads.  Every wait is
+// bounded (see tc_gemm.cuh); on a time-out the copy thread waits, again bounded, for the copies it
+// has in flight before the CTA returns.
+#pragma once
+#include <cuda.h>
+
+#include "tc_gemm.cuh"
+
+namespace dynbatch {
+namespace tcg {
+
+constexpr int kTileM = 128;            // features per CTA = tensor-memory lanes
+constexpr int kTileN = 64;             // classes per CTA = accumulator columns
+constexpr int kChunk = 32;             // fp32 per 128-byte swizzled row
+constexpr int kStepRows = 8;           // reduction depth of one TF32 product
+constexpr int kRowsPerStage = 32;      // samples per stage: four products' worth
+constexpr int kStages = 2;
+constexpr int kChunkBytes = kRowsPerStage * 128;            // one [32 x 32] box
+constexpr int kAChunks = kTileM / kChunk, kBChunks = kTileN / kChunk;
+constexpr int kABytes = kAChunks * kChunkBytes;             // X_hi (or X_lo) part of a stage
+constexpr int kBBytes = kBChunks * kChunkBytes;             // E_hi (or E_lo) part of a stage
+constexpr int kStageBytes = 2 * kABytes + 2 * kBBytes;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024;    // + slack for 1024-byte alignment
+constexpr int kEpilogueWarps = 4;
+constexpr int kEpilogueThreads = kEpilogueWarps * 32;
+constexpr int kThreads = 64 + kEpilogueThreads;
+constexpr int kMaxAcc = 512 / kTileN - 1;                   // main accumulators beside the cross-term one
+constexpr int kStagePitch = kTileN + 4;                     // floats per row of the output staging tile
+static_assert(kTileM * kStagePitch * 4 <= kStages * kStageBytes, "output staging fits in the operand stages");
+
+struct GradArgs {
+    CUtensorMap x_hi, x_lo;        // [padded rows, D], boxes of 32 x 32, 128-byte swizzle of 32-byte pieces
+    CUtensorMap e_hi, e_lo;        // [padded rows, C]
+    float* out[DB_MAX_K];          // G_w, [D, C] row-major
+    int row0[DB_MAX_K];            // first row of worker w in the split arrays (multiple of 8)
+    int steps[DB_MAX_K];           // its padded row count / 8
+    int D, C;
+    int n_acc;                     // main accumulators in use, 1..kMaxAcc
+    int* status;
+};
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(tc::smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+// One box of a 2-D tensor map into shared memory; x counts elements of the contiguous dimension and
+// must be a multiple of 4 (16 bytes).  Coordinates outside the tensor read as zero.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(tc::smem_u32(bar)) : "memory");
+}
+
+// Shared-memory matrix descriptor of an operand stored output-index-major.  For 32-bit elements the
+// tensor core accepts this orientation only with the 128-byte swizzle that permutes 32-byte pieces
+// (layout type 1; the TMA mode of the same name writes it): 32 consecutive output indices form a
+// 128-byte row, 4 reduction rows a 512-byte swizzle group.  The next 32 output indices start
+// kChunkBytes further (leading byte offset), the next 4 reduction rows 512 bytes further (stride
+// byte offset); one product consumes two such groups.
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>(kChunkBytes >> 4) << 16;
+    d |= static_cast<uint64_t>(512 >> 4) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    d |= static_cast<uint64_t>(1) << 61;
+    return d;
+}
+// fp32 accumulator, TF32 operands, both output-index-major (bits 15 and 16), M x N tile.
+__host__ __device__ constexpr uint32_t instr_desc_tf32_mn(int M, int N) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | (1u << 16) | (static_cast<uint32_t>(N >> 3) << 17) |
+           (static_cast<uint32_t>(M >> 4) << 24);
+}
+
+// grid: (ceil(C / 64), ceil(D / 128), workers)
+__global__ void __launch_bounds__(kThreads)
+grad_tma_kernel(const __grid_constant__ GradArgs g) {
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kStages];
+    __shared__ __align__(8) uint64_t empty_bar[kStages];
+    __shared__ __align__(8) uint64_t done_bar;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ volatile int abort_flag;
+
+    unsigned char* tiles = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int z = blockIdx.z;
+    const int m0 = blockIdx.y * kTileM, n0 = blockIdx.x * kTileN;
+    const int steps = g.steps[z];
+    const int loads = (steps * kStepRows + kRowsPerStage - 1) / kRowsPerStage;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < kStages; ++s) {
+            tc::mbar_init(&full_bar[s], 1);
+            tc::mbar_init(&empty_bar[s], 1);
+        }
+        tc::mbar_init(&done_bar, 1);
+        tc::fence_barrier_init();
+    }
+    const uint32_t tmem_cols = tc::tmem_columns((g.n_acc + 1) * kTileN);
+    if (warp == 1) tc::tmem_alloc(&tmem_base_slot, tmem_cols);
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    // everything above overlaps the kernel that writes the split operands
+    tc::griddep_launch_dependents();
+    tc::griddep_wait();
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA copies
+        if (lane == 0) {
+            int issued = 0;
+            for (int l = 0; l < loads; ++l) {
+                const int s = l % kStages;
+                if (l >= kStages &&
+                    !tc::mbar_wait(&empty_bar[s], ((l / kStages) - 1) & 1, &abort_flag, g.status, 4))
+                    break;
+                if (abort_flag) break;
+                mbar_expect_tx(&full_bar[s], kStageBytes);
+                const uint32_t dst = tc::smem_u32(tiles + s * kStageBytes);
+                const int row = g.row0[z] + l * kRowsPerStage;
+#pragma unroll
+                for (int c = 0; c < kAChunks; ++c) {
+                    tma_load_2d(dst + c * kChunkBytes, &g.x_hi, m0 + c * kChunk, row, &full_bar[s]);
+                    tma_load_2d(dst + kABytes + c * kChunkBytes, &g.x_lo, m0 + c * kChunk, row, &full_bar[s]);
+                }
+#pragma unroll
+                for (int c = 0; c < kBChunks; ++c) {
+                    tma_load_2d(dst + 2 * kABytes + c * kChunkBytes, &g.e_hi, n0 + c * kChunk, row, &full_bar[s]);
+                    tma_load_2d(dst + 2 * kABytes + kBBytes + c * kChunkBytes, &g.e_lo, n0 + c * kChunk, row,
+                                &full_bar[s]);
+                }
+                issued = l + 1;
+            }
+            // the copies issued last write into this CTA's shared memory until they land: see them
+            // complete (bounded) before this thread lets the CTA exit, whatever the other roles do
+            for (int l = max(0, issued - kStages); l < issued; ++l) {
+                const unsigned long long t0 = tc::global_ns();
+                while (!tc::mbar_try_wait(&full_bar[l % kStages], (l / kStages) & 1) &&
+                       tc::global_ns() - t0 < tc::kWaitLimitNs) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ tensor-core issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_tf32_mn(kTileM, kTileN);
+            const uint32_t acc_cross = tmem_base + g.n_acc * kTileN;
+            bool alive = true;
+            for (int l = 0; l < loads && alive; ++l) {
+                const int s = l % kStages;
+                alive = tc::mbar_wait(&full_bar[s], (l / kStages) & 1, &abort_flag, g.status, 5);
+                if (!alive) break;
+                tc::tc_fence_after();
+                const uint32_t st = tc::smem_u32(tiles + s * kStageBytes);
+                const uint32_t acc_main = tmem_base + (l % g.n_acc) * kTileN;
+                const int here = min(kRowsPerStage / kStepRows, steps - l * (kRowsPerStage / kStepRows));
+                for (int q = 0; q < here; ++q) {
+                    const uint32_t off = q * 1024;      // 8 rows of 128 bytes
+                    const uint64_t a_hi = smem_desc_mn_sw128(st + off);
+                    const uint64_t a_lo = smem_desc_mn_sw128(st + kABytes + off);
+                    const uint64_t b_hi = smem_desc_mn_sw128(st + 2 * kABytes + off);
+                    const uint64_t b_lo = smem_desc_mn_sw128(st + 2 * kABytes + kBBytes + off);
+                    tc::mma_tf32(acc_cross, a_lo, b_hi, idesc, (l | q) != 0);
+                    tc::mma_tf32(acc_cross, a_hi, b_lo, idesc, 1);
+                    tc::mma_tf32(acc_main, a_hi, b_hi, idesc, (l >= g.n_acc) || q != 0);
+                }
+                tc::mma_commit(&empty_bar[s]);
+            }
+            tc::mma_commit(&done_bar);
+            if (!alive) {
+                const unsigned long long t0 = tc::global_ns();
+                while (!tc::mbar_try_wait(&done_bar, 0) && tc::global_ns() - t0 < tc::kWaitLimitNs) {}
+            }
+            tc::tc_fence_before();
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue
+        const bool alive = tc::mbar_wait(&done_bar, 0, &abort_flag, g.status, 6);
+        tc::tc_fence_after();
+        const int et = tid - 64;                     // 0..127
+        const int quarter = warp & 3;                // the tensor-memory lanes this warp may read
+        if (alive) {
+            const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+            const int used = min(g.n_acc, loads);
+            float* srow = reinterpret_cast<float*>(tiles) + (quarter * 32 + lane) * kStagePitch;
+#pragma unroll 1
+            for (int c0 = 0; c0 < kTileN; c0 += 32) {
+                uint32_t r[32], x[32];
+                __syncwarp();
+                tc::tmem_load32(lane_base + g.n_acc * kTileN + c0, r);
+                for (int a = used - 1; a >= 0; --a) {
+                    tc::tmem_load32(lane_base + a * kTileN + c0, x);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(x[j]));
+                }
+#pragma unroll
+                for (int j = 0; j < 32; j += 4)
+                    *reinterpret_cast<float4*>(srow + c0 + j) =
+                        make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                                    __uint_as_float(r[j + 3]));
+            }
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
+        if (alive) {
+            // whole rows of the tile, 16 threads per row
+            const float* stage = reinterpret_cast<const float*>(tiles);
+            float* obase = g.out[z];
+            const int rows = min(kTileM, g.D - m0), cols = min(kTileN, g.C - n0);
+            constexpr int kVecPerRow = kTileN / 4;
+            constexpr int kRowsPerPass = kEpilogueThreads / kVecPerRow;
+            const int vcol = (et % kVecPerRow) * 4, rsub = et / kVecPerRow;
+            const bool vec_ok = (g.C % 4 == 0) && (reinterpret_cast<uintptr_t>(obase) % 16 == 0);
+            for (int r0 = 0; r0 < rows; r0 += kRowsPerPass) {
+                const int rr = r0 + rsub;
+                if (rr >= rows || vcol >= cols) continue;
+                const float4 val = *reinterpret_cast<const float4*>(stage + rr * kStagePitch + vcol);
+                float* dst = obase + static_cast<long long>(m0 + rr) * g.C + n0 + vcol;
+                if (vec_ok && vcol + 4 <= cols) {
+                    *reinterpret_cast<float4*>(dst) = val;
+                } else {
+                    dst[0] = val.x;
+                    if (vcol + 1 < cols) dst[1] = val.y;
+                    if (vcol + 2 < cols) dst[2] = val.z;
+                    if (vcol + 3 < cols) dst[3] = val.w;
+                }
+            }
+        }
+        tc::tc_fence_before();
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tc::tc_fence_after();
+        tc::tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+}  // namespace tcg
+}  // namespace dynbatch

@@ -11,13 +11,17 @@
 //      the last CTA of a worker also folds the per-sample losses into the mean;
 //   3. gradient: G = X^T E, reduction depth b_i.
 // The two contractions run on the tensor cores (tcgen05, three TF32 products per
-// fp32 product, see tc_gemm.cuh).  An fp32 FFMA version on shared-memory tiles is
+// fp32 product).  The logits use the general contraction of tc_gemm.cuh, which
+// converts fp32 operands on the fly; for the gradient the softmax kernel leaves E
+// and a copy of X already split into TF32 halves, row-major, and the contraction of
+// tc_grad.cuh reads them with TMA.  An fp32 FFMA version on shared-memory tiles is
 // kept as the accuracy reference and for very large b_i.
 #include <algorithm>
 #include <cstdint>
 
 #include "common.h"
 #include "tc_gemm.cuh"
+#include "tc_grad.cuh"
 
 namespace dynbatch {
 namespace {
@@ -162,21 +166,72 @@ __device__ __forceinline__ float block_reduce(float x, float* smem, bool take_ma
 struct RowGroups {
     int K;
     int off[DB_MAX_K + 1];
+    int poff[DB_MAX_K + 1];   // SPLIT: the workers' first rows in the split arrays (multiples of 8)
 };
 
-template <bool IN_REGS>
+// SPLIT: where the operands of the tensor-core gradient contraction go.  Row i of worker w lands in
+// row poff[w] + (i - off[w]) of four row-major arrays: E split into TF32 halves (e_hi + e_lo = E up to
+// 2^-22) and the same split of the sample's feature row X[i, :].  The grid then has one CTA per row of
+// the split arrays; the CTAs of the up to 7 padding rows behind each worker write zeros.
+struct SplitOut {
+    float* e_hi;
+    float* e_lo;
+    long long e_pitch;     // floats per row, >= C
+    const float* X;        // [rows, D] row-major
+    float* x_hi;
+    float* x_lo;
+    long long x_pitch;     // floats per row, >= D, multiple of 4
+    int D;
+    int x_vec;             // D % 4 == 0 and X 16-byte aligned: 128-bit loads
+};
+
+template <bool IN_REGS, bool SPLIT>
 __global__ void __launch_bounds__(kThreads)
 softmax_residual_kernel(const float* __restrict__ partials, int splits, long long split_stride,
                         const int32_t* __restrict__ y, float* __restrict__ E, float* __restrict__ row_loss,
                         const __grid_constant__ RowGroups groups, int C, unsigned int* __restrict__ tickets,
-                        float* __restrict__ losses) {
+                        float* __restrict__ losses, const __grid_constant__ SplitOut so) {
     __shared__ float smem[kThreads / 32];
     __shared__ float z_label;
     __shared__ bool is_last;
     tc::griddep_launch_dependents();
-    const int i = blockIdx.x;
-    int w = 0;
-    while (w + 1 < groups.K && i >= groups.off[w + 1]) ++w;
+    int i = blockIdx.x, w = 0;
+    float* eh = nullptr;
+    float* el = nullptr;
+    if (SPLIT) {
+        const int ip = blockIdx.x;
+        while (w + 1 < groups.K && ip >= groups.poff[w + 1]) ++w;
+        const int r = ip - groups.poff[w];
+        eh = so.e_hi + static_cast<long long>(ip) * so.e_pitch;
+        el = so.e_lo + static_cast<long long>(ip) * so.e_pitch;
+        float* xh = so.x_hi + static_cast<long long>(ip) * so.x_pitch;
+        float* xl = so.x_lo + static_cast<long long>(ip) * so.x_pitch;
+        if (r >= groups.off[w + 1] - groups.off[w]) {
+            // padding row: zeros in all four arrays (the workspace may hold anything, NaN included)
+            for (int c = threadIdx.x; c < C; c += kThreads) { eh[c] = 0.0f; el[c] = 0.0f; }
+            for (int d = threadIdx.x; d < so.D; d += kThreads) { xh[d] = 0.0f; xl[d] = 0.0f; }
+            return;
+        }
+        i = groups.off[w] + r;
+        // the feature row is an input of the whole call, not of the logits kernel: split it while that runs
+        const float* xr = so.X + static_cast<long long>(i) * so.D;
+        if (so.x_vec) {
+            for (int d = threadIdx.x * 4; d < so.D; d += 4 * kThreads) {
+                const float4 v = __ldg(reinterpret_cast<const float4*>(xr + d));
+                float4 h, l;
+                tc::split_tf32(v.x, h.x, l.x);
+                tc::split_tf32(v.y, h.y, l.y);
+                tc::split_tf32(v.z, h.z, l.z);
+                tc::split_tf32(v.w, h.w, l.w);
+                *reinterpret_cast<float4*>(xh + d) = h;
+                *reinterpret_cast<float4*>(xl + d) = l;
+            }
+        } else {
+            for (int d = threadIdx.x; d < so.D; d += kThreads) tc::split_tf32(__ldg(xr + d), xh[d], xl[d]);
+        }
+    } else {
+        while (w + 1 < groups.K && i >= groups.off[w + 1]) ++w;
+    }
     const int row0 = groups.off[w], b = groups.off[w + 1] - row0;
     unsigned int* ticket = tickets + w;
     float* loss = losses ? losses + w : nullptr;
@@ -246,14 +301,18 @@ softmax_residual_kernel(const float* __restrict__ partials, int splits, long lon
             if (c < C) {
                 float r = z[j] / den;
                 if (c == label) r -= 1.0f;
-                e[c] = r * inv_b;
+                r *= inv_b;
+                if (SPLIT) tc::split_tf32(r, eh[c], el[c]);
+                else e[c] = r;
             }
         }
     } else {
         for (int c = threadIdx.x; c < C; c += kThreads) {
             float r = expf(e[c] - zmax) / den;
             if (c == label) r -= 1.0f;
-            e[c] = r * inv_b;
+            r *= inv_b;
+            if (SPLIT) tc::split_tf32(r, eh[c], el[c]);
+            else e[c] = r;
         }
     }
     if (loss == nullptr) return;
@@ -287,16 +346,17 @@ struct OverlappedLaunch {
     }
 };
 
+// `split` non-null: one CTA per row of the split arrays (groups.poff[groups.K] of them), else one per sample.
 db_status launch_softmax(const float* partials, int splits, long long split_stride, const int32_t* y, float* E,
                          float* row_loss, const RowGroups& groups, int rows, int C, unsigned int* tickets,
-                         float* losses, cudaStream_t stream, bool overlap) {
-    OverlappedLaunch L(dim3(rows), dim3(kThreads), 0, stream, overlap);
-    if (C <= 4 * kThreads)
-        DB_CUDA_TRY(cudaLaunchKernelEx(&L.cfg, softmax_residual_kernel<true>, partials, splits, split_stride, y, E,
-                                       row_loss, groups, C, tickets, losses));
-    else
-        DB_CUDA_TRY(cudaLaunchKernelEx(&L.cfg, softmax_residual_kernel<false>, partials, splits, split_stride, y, E,
-                                       row_loss, groups, C, tickets, losses));
+                         float* losses, cudaStream_t stream, bool overlap, const SplitOut* split = nullptr) {
+    const bool in_regs = C <= 4 * kThreads;
+    OverlappedLaunch L(dim3(split ? groups.poff[groups.K] : rows), dim3(kThreads), 0, stream, overlap);
+    const SplitOut so = split ? *split : SplitOut{};
+    auto fn = split ? (in_regs ? softmax_residual_kernel<true, true> : softmax_residual_kernel<false, true>)
+                    : (in_regs ? softmax_residual_kernel<true, false> : softmax_residual_kernel<false, false>);
+    DB_CUDA_TRY(cudaLaunchKernelEx(&L.cfg, fn, partials, splits, split_stride, y, E, row_loss, groups, C, tickets,
+                                   losses, so));
     return DB_OK;
 }
 
@@ -316,36 +376,20 @@ int logit_splits(int b, int D, int C) {
 constexpr int kMaxTensorCoreBatch = 4096;  // longer reductions over the batch go to FFMA
 constexpr size_t kStatusBytes = 16;        // device status word of the tensor-core kernels
 
+// Workspace of the FFMA path (one worker).
 struct WorkerLayout {
-    bool tensor;            // tensor-core path
     int splits, k_per_split;
-    int n_tile;             // accumulator columns of the logits GEMM (tensor path)
     size_t partial_bytes, e_bytes, loss_bytes;
     size_t total() const { return kStatusBytes + partial_bytes + e_bytes + loss_bytes; }
 };
 
-WorkerLayout layout_for(int b, int D, int C, bool tensor) {
+WorkerLayout layout_for(int b, int D, int C) {
     WorkerLayout L;
-    L.tensor = tensor;
-    L.n_tile = b <= 32 ? 32 : (b <= 64 ? 64 : 128);
-    if (tensor) {
-        // logits are computed transposed: 128 classes x n_tile samples per CTA, split over D so that
-        // about one CTA per SM exists; splits are whole 32-feature blocks
-        const long long tiles = static_cast<long long>((C + tc::kTileM - 1) / tc::kTileM) * ((b + L.n_tile - 1) / L.n_tile);
-        long long s = sm_count() / tiles;
-        const int kblocks = (D + tc::kBlockK - 1) / tc::kBlockK;
-        if (s > kblocks) s = kblocks;
-        if (s < 1) s = 1;
-        const int per_blocks = static_cast<int>((kblocks + s - 1) / s);
-        L.k_per_split = per_blocks * tc::kBlockK;
-        L.splits = (D + L.k_per_split - 1) / L.k_per_split;
-    } else {
-        L.splits = logit_splits(b, D, C);
-        int per = (D + L.splits - 1) / L.splits;
-        per = (per + kDepth - 1) / kDepth * kDepth;  // whole stages, keeps 16-byte alignment of k offsets
-        L.k_per_split = per;
-        L.splits = (D + per - 1) / per;
-    }
+    L.splits = logit_splits(b, D, C);
+    int per = (D + L.splits - 1) / L.splits;
+    per = (per + kDepth - 1) / kDepth * kDepth;  // whole stages, keeps 16-byte alignment of k offsets
+    L.k_per_split = per;
+    L.splits = (D + per - 1) / per;
     L.partial_bytes = round16(sizeof(float) * static_cast<size_t>(L.splits) * b * C);
     L.e_bytes = round16(sizeof(float) * static_cast<size_t>(b) * C);
     L.loss_bytes = round16(sizeof(float) * static_cast<size_t>(b));
@@ -355,32 +399,22 @@ WorkerLayout layout_for(int b, int D, int C, bool tensor) {
 bool valid_shape(int b, int D, int C) { return b >= 1 && b <= 65535 && D >= 1 && C >= 1; }
 
 using TcKernel = void (*)(const tc::GemmArgs);
-using TcGroupedKernel = void (*)(const tc::GemmArgs, const tc::GroupArgs);
 
 template <int N_TILE, int MODE_A>
-void pick_tc_b(int mode_b, TcKernel* single, TcGroupedKernel* grouped) {
+TcKernel pick_tc_b(int mode_b) {
     switch (mode_b) {
-        case tc::kLoadKVec:
-            *single = tc::tf32x3_gemm_kernel<N_TILE, MODE_A, tc::kLoadKVec>;
-            *grouped = tc::tf32x3_gemm_grouped_kernel<N_TILE, MODE_A, tc::kLoadKVec>;
-            break;
-        case tc::kLoadRowVec:
-            *single = tc::tf32x3_gemm_kernel<N_TILE, MODE_A, tc::kLoadRowVec>;
-            *grouped = tc::tf32x3_gemm_grouped_kernel<N_TILE, MODE_A, tc::kLoadRowVec>;
-            break;
-        default:
-            *single = tc::tf32x3_gemm_kernel<N_TILE, MODE_A, tc::kLoadScalar>;
-            *grouped = tc::tf32x3_gemm_grouped_kernel<N_TILE, MODE_A, tc::kLoadScalar>;
-            break;
+        case tc::kLoadKVec: return tc::tf32x3_gemm_kernel<N_TILE, MODE_A, tc::kLoadKVec>;
+        case tc::kLoadRowVec: return tc::tf32x3_gemm_kernel<N_TILE, MODE_A, tc::kLoadRowVec>;
+        default: return tc::tf32x3_gemm_kernel<N_TILE, MODE_A, tc::kLoadScalar>;
     }
 }
 
 template <int N_TILE>
-void pick_tc(int mode_a, int mode_b, TcKernel* single, TcGroupedKernel* grouped) {
+TcKernel pick_tc(int mode_a, int mode_b) {
     switch (mode_a) {
-        case tc::kLoadKVec: pick_tc_b<N_TILE, tc::kLoadKVec>(mode_b, single, grouped); break;
-        case tc::kLoadRowVec: pick_tc_b<N_TILE, tc::kLoadRowVec>(mode_b, single, grouped); break;
-        default: pick_tc_b<N_TILE, tc::kLoadScalar>(mode_b, single, grouped); break;
+        case tc::kLoadKVec: return pick_tc_b<N_TILE, tc::kLoadKVec>(mode_b);
+        case tc::kLoadRowVec: return pick_tc_b<N_TILE, tc::kLoadRowVec>(mode_b);
+        default: return pick_tc_b<N_TILE, tc::kLoadScalar>(mode_b);
     }
 }
 
@@ -392,58 +426,37 @@ int load_mode(const float* p, long long row_stride, long long k_stride) {
     return tc::kLoadScalar;
 }
 
-int weaker_mode(int a, int b) { return a == b ? a : tc::kLoadScalar; }
-
 // out(m, n) = sum_k A(m, k) B(n, k) on the tensor cores; a.k_per_split must be a multiple of 32.
-// With `groups` (n_groups problems sharing strides, M and N) blockIdx.z selects the problem.
-db_status launch_tc_gemm(tc::GemmArgs a, int n_tile, cudaStream_t stream, const tc::GroupArgs* groups = nullptr,
-                         int n_groups = 0, bool overlap = false) {
+db_status launch_tc_gemm(tc::GemmArgs a, int n_tile, cudaStream_t stream, bool overlap = false) {
     if (n_tile != 32 && n_tile != 64) n_tile = 128;
-    int mode_a, mode_b, max_k = a.K;
-    if (groups) {
-        mode_a = load_mode(groups->A[0], a.a_row, a.a_k);
-        mode_b = load_mode(groups->B[0], a.b_row, a.b_k);
-        max_k = 0;
-        for (int z = 0; z < n_groups; ++z) {
-            mode_a = weaker_mode(mode_a, load_mode(groups->A[z], a.a_row, a.a_k));
-            mode_b = weaker_mode(mode_b, load_mode(groups->B[z], a.b_row, a.b_k));
-            if (groups->K[z] > max_k) max_k = groups->K[z];
-        }
-        a.k_per_split = (max_k + tc::kBlockK - 1) / tc::kBlockK * tc::kBlockK;
-    } else {
-        mode_a = load_mode(a.A, a.a_row, a.a_k);
-        mode_b = load_mode(a.B, a.b_row, a.b_k);
-    }
+    const int mode_a = load_mode(a.A, a.a_row, a.a_k), mode_b = load_mode(a.B, a.b_row, a.b_k);
     // one main accumulator per four reduction blocks (chains of 16 additions), within 512 columns
     const int blocks = a.k_per_split / tc::kBlockK;
     int n_acc = (blocks + 3) / 4;
     if (n_acc > 512 / n_tile - 1) n_acc = 512 / n_tile - 1;
     a.n_acc = n_acc < 1 ? 1 : n_acc;
     TcKernel fn = nullptr;
-    TcGroupedKernel gfn = nullptr;
     int smem;
     switch (n_tile) {
-        case 32: pick_tc<32>(mode_a, mode_b, &fn, &gfn); smem = tc::SmemLayout<32>::kBytes; break;
-        case 64: pick_tc<64>(mode_a, mode_b, &fn, &gfn); smem = tc::SmemLayout<64>::kBytes; break;
-        default: pick_tc<128>(mode_a, mode_b, &fn, &gfn); smem = tc::SmemLayout<128>::kBytes; break;
+        case 32: fn = pick_tc<32>(mode_a, mode_b); smem = tc::SmemLayout<32>::kBytes; break;
+        case 64: fn = pick_tc<64>(mode_a, mode_b); smem = tc::SmemLayout<64>::kBytes; break;
+        default: fn = pick_tc<128>(mode_a, mode_b); smem = tc::SmemLayout<128>::kBytes; break;
     }
-    if (groups) {
-        DB_CUDA_TRY(cudaFuncSetAttribute(gfn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        dim3 grid((a.N + n_tile - 1) / n_tile, (a.M + tc::kTileM - 1) / tc::kTileM, n_groups);
-        OverlappedLaunch L(grid, dim3(tc::kThreads), smem, stream, overlap);
-        DB_CUDA_TRY(cudaLaunchKernelEx(&L.cfg, gfn, a, *groups));
-    } else {
-        DB_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        const int splits = a.k_per_split > 0 ? (a.K + a.k_per_split - 1) / a.k_per_split : 1;
-        dim3 grid((a.N + n_tile - 1) / n_tile, (a.M + tc::kTileM - 1) / tc::kTileM, splits < 1 ? 1 : splits);
-        OverlappedLaunch L(grid, dim3(tc::kThreads), smem, stream, overlap);
-        DB_CUDA_TRY(cudaLaunchKernelEx(&L.cfg, fn, a));
-    }
+    DB_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    const int splits = a.k_per_split > 0 ? (a.K + a.k_per_split - 1) / a.k_per_split : 1;
+    dim3 grid((a.N + n_tile - 1) / n_tile, (a.M + tc::kTileM - 1) / tc::kTileM, splits < 1 ? 1 : splits);
+    OverlappedLaunch L(grid, dim3(tc::kThreads), smem, stream, overlap);
+    DB_CUDA_TRY(cudaLaunchKernelEx(&L.cfg, fn, a));
     DB_CUDA_TRY(cudaGetLastError());
     return DB_OK;
 }
 
 bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
+
+// defined below, beside the grouped entry point
+size_t grouped_workspace_total(long long rows, int K, int D, int C);
+db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, const int32_t* offsets, int K, int D,
+                             int C, float* const* G, float* losses, void* workspace, cudaStream_t stream);
 
 }  // namespace
 }  // namespace dynbatch
@@ -471,8 +484,10 @@ extern "C" db_status db_contract_f32(const float* A, int64_t a_row, int64_t a_k,
 extern "C" size_t db_worker_grad_workspace_bytes(int32_t b_i, int32_t D, int32_t C) {
     using namespace dynbatch;
     if (!valid_shape(b_i, D, C)) return 0;
-    const size_t a = layout_for(b_i, D, C, true).total(), f = layout_for(b_i, D, C, false).total();
-    return a > f ? a : f;
+    const size_t f = layout_for(b_i, D, C).total();
+    if (b_i > kMaxTensorCoreBatch) return f;
+    const size_t t = grouped_workspace_total(b_i, 1, D, C);
+    return t > f ? t : f;
 }
 
 extern "C" db_status db_worker_grad_ex(const float* X, const int32_t* y, const float* W, int32_t b_i,
@@ -484,9 +499,14 @@ extern "C" db_status db_worker_grad_ex(const float* X, const int32_t* y, const f
     if (flags & ~static_cast<uint32_t>(DB_WORKER_GRAD_FFMA)) return DB_ERR_ARG;
     if (reinterpret_cast<uintptr_t>(workspace) % 16) return DB_ERR_ARG;
     if (workspace_bytes < db_worker_grad_workspace_bytes(b_i, D, C)) return DB_ERR_ARG;
-    const bool tensor = !(flags & DB_WORKER_GRAD_FFMA) && b_i <= kMaxTensorCoreBatch;
-    const WorkerLayout L = layout_for(b_i, D, C, tensor);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (!(flags & DB_WORKER_GRAD_FFMA) && b_i <= kMaxTensorCoreBatch) {
+        // the tensor-core path is the grouped one with a single worker
+        const int32_t offsets[2] = {0, b_i};
+        float* const out[1] = {G};
+        return worker_grad_tensor(X, y, W, offsets, 1, D, C, out, loss, workspace, stream);
+    }
+    const WorkerLayout L = layout_for(b_i, D, C);
 
     char* base = static_cast<char*>(workspace);
     int* status = reinterpret_cast<int*>(base);
@@ -497,15 +517,7 @@ extern "C" db_status db_worker_grad_ex(const float* X, const int32_t* y, const f
     DB_CUDA_TRY(cudaMemsetAsync(status, 0, kStatusBytes, stream));
 
     // 1. logits, split over D
-    if (tensor) {
-        tc::GemmArgs a{};
-        a.A = W; a.a_row = 1; a.a_k = C;          // A(m = class, k = feature) = W[k, m]
-        a.B = X; a.b_row = D; a.b_k = 1;          // B(n = sample, k = feature) = X[n, k]
-        a.out = partials; a.o_m = 1; a.o_n = C; a.o_split = bc;   // Z[n, m], one slab per split
-        a.M = C; a.N = b_i; a.K = D; a.k_per_split = L.k_per_split; a.status = status;
-        const db_status st = launch_tc_gemm(a, L.n_tile, stream);
-        if (st != DB_OK) return st;
-    } else {
+    {
         const bool vec4 = (D % 4 == 0) && (C % 4 == 0) && aligned16(X) && aligned16(W);
         dim3 grid((C + kTile - 1) / kTile, (b_i + kTile - 1) / kTile, L.splits);
         if (vec4)
@@ -522,23 +534,12 @@ extern "C" db_status db_worker_grad_ex(const float* X, const int32_t* y, const f
     one.off[0] = 0;
     one.off[1] = b_i;
     {
-        // after the tensor-core logits kernel the softmax may start early (it waits for the partials itself)
         const db_status st = launch_softmax(partials, L.splits, bc, y, E, row_loss, one, b_i, C,
-                                            reinterpret_cast<unsigned int*>(status) + 1, loss, stream, tensor);
+                                            reinterpret_cast<unsigned int*>(status) + 1, loss, stream, false);
         if (st != DB_OK) return st;
     }
     // 3. G = X^T E
-    if (tensor) {
-        tc::GemmArgs a{};
-        a.A = X; a.a_row = 1; a.a_k = D;          // A(m = feature, k = sample) = X[k, m]
-        a.B = E; a.b_row = 1; a.b_k = C;          // B(n = class, k = sample) = E[k, n]
-        a.out = G; a.o_m = C; a.o_n = 1; a.o_split = 0;
-        a.M = D; a.N = C; a.K = b_i;
-        a.k_per_split = (b_i + tc::kBlockK - 1) / tc::kBlockK * tc::kBlockK;   // one split
-        a.status = status;
-        const db_status st = launch_tc_gemm(a, 64, stream, nullptr, 0, true);
-        if (st != DB_OK) return st;
-    } else {
+    {
         const bool vec4 = (D % 4 == 0) && (C % 4 == 0) && aligned16(X) && aligned16(G);
         dim3 grid((C + kTile - 1) / kTile, (D + kTile - 1) / kTile, 1);
         if (vec4)
@@ -555,9 +556,15 @@ namespace {
 
 struct GroupedLayout {
     int splits, k_per_split, n_tile;
-    size_t header_bytes, partial_bytes, e_bytes, loss_bytes;
-    size_t total() const { return header_bytes + partial_bytes + e_bytes + loss_bytes; }
+    long long rows_p;            // rows of the split arrays: every worker padded to a multiple of 8 (upper bound)
+    long long x_pitch, e_pitch;  // floats per row of the split arrays (multiples of 32: 128-byte rows)
+    size_t header_bytes, partial_bytes, e_bytes, loss_bytes, xs_bytes, es_bytes;
+    size_t total() const {
+        return header_bytes + partial_bytes + e_bytes + loss_bytes + 2 * xs_bytes + 2 * es_bytes;
+    }
 };
+
+long long round_up(long long x, long long m) { return (x + m - 1) / m * m; }
 
 // All workers' rows go through one logits contraction (they share W); split over D for about one CTA per SM.
 GroupedLayout grouped_layout(long long rows, int K, int D, int C) {
@@ -571,15 +578,146 @@ GroupedLayout grouped_layout(long long rows, int K, int D, int C) {
     const int per_blocks = static_cast<int>((kblocks + s - 1) / s);
     L.k_per_split = per_blocks * tc::kBlockK;
     L.splits = (D + L.k_per_split - 1) / L.k_per_split;
+    L.rows_p = round_up(rows + 7LL * K, 8);
+    L.x_pitch = round_up(D, 32);
+    L.e_pitch = round_up(C, 32);
     L.header_bytes = round16(kStatusBytes + sizeof(unsigned int) * static_cast<size_t>(K));
     L.partial_bytes = round16(sizeof(float) * static_cast<size_t>(L.splits) * rows * C);
     L.e_bytes = round16(sizeof(float) * static_cast<size_t>(rows) * C);
     L.loss_bytes = round16(sizeof(float) * static_cast<size_t>(rows));
+    L.xs_bytes = sizeof(float) * static_cast<size_t>(L.rows_p) * L.x_pitch;
+    L.es_bytes = sizeof(float) * static_cast<size_t>(L.rows_p) * L.e_pitch;
     return L;
 }
 
+size_t grouped_workspace_total(long long rows, int K, int D, int C) { return grouped_layout(rows, K, D, C).total(); }
+
 bool valid_group_shape(long long rows, int K, int D, int C) {
     return K >= 1 && K <= DB_MAX_K && rows >= K && rows <= (1 << 22) && D >= 1 && C >= 1;
+}
+
+// cuTensorMapEncodeTiled, looked up through the runtime so that the library needs no link against the driver.
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+        if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &p, 12000, cudaEnableDefault, &q) !=
+                cudaSuccess || q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// Tensor map of a row-major fp32 array [rows, cols] with `pitch` floats per row, read in boxes of
+// 32 rows x 32 columns with the 128-byte swizzle of 32-byte pieces (the only one the tensor core takes
+// for 32-bit operands that are contiguous along the output index); elements outside [rows, cols] read as zero.
+db_status make_operand_map(CUtensorMap* map, float* base, long long rows, long long cols, long long pitch) {
+    EncodeTiledFn enc = encode_tiled();
+    if (!enc) {
+        record_message("cuTensorMapEncodeTiled is not available from this driver");
+        return DB_ERR_CUDA;
+    }
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(pitch) * sizeof(float)};
+    const cuuint32_t box[2] = {tcg::kChunk, tcg::kRowsPerStage};
+    const cuuint32_t elem[2] = {1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, elem,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        record_message("cuTensorMapEncodeTiled rejected the operand layout of the gradient contraction");
+        return DB_ERR_CUDA;
+    }
+    return DB_OK;
+}
+
+// The tensor-core path for K >= 1 workers; arguments already validated.
+db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, const int32_t* offsets, int K, int D,
+                             int C, float* const* G, float* losses, void* workspace, cudaStream_t stream) {
+    const long long rows = offsets[K];
+    const GroupedLayout L = grouped_layout(rows, K, D, C);
+    char* base = static_cast<char*>(workspace);
+    int* status = reinterpret_cast<int*>(base);
+    unsigned int* tickets = reinterpret_cast<unsigned int*>(base + kStatusBytes);
+    char* cur = base + L.header_bytes;
+    float* partials = reinterpret_cast<float*>(cur); cur += L.partial_bytes;
+    float* E = reinterpret_cast<float*>(cur); cur += L.e_bytes;
+    float* row_loss = reinterpret_cast<float*>(cur); cur += L.loss_bytes;
+    float* x_hi = reinterpret_cast<float*>(cur); cur += L.xs_bytes;
+    float* x_lo = reinterpret_cast<float*>(cur); cur += L.xs_bytes;
+    float* e_hi = reinterpret_cast<float*>(cur); cur += L.es_bytes;
+    float* e_lo = reinterpret_cast<float*>(cur);
+    const long long rc = rows * C;
+
+    RowGroups rg{};
+    rg.K = K;
+    for (int w = 0; w <= K; ++w) rg.off[w] = offsets[w];
+    rg.poff[0] = 0;
+    for (int w = 0; w < K; ++w) rg.poff[w + 1] = rg.poff[w] + static_cast<int>(round_up(offsets[w + 1] - offsets[w], 8));
+    const long long rows_p = rg.poff[K];
+
+    tcg::GradArgs ga{};
+    db_status st;
+    if ((st = make_operand_map(&ga.x_hi, x_hi, rows_p, D, L.x_pitch)) != DB_OK) return st;
+    if ((st = make_operand_map(&ga.x_lo, x_lo, rows_p, D, L.x_pitch)) != DB_OK) return st;
+    if ((st = make_operand_map(&ga.e_hi, e_hi, rows_p, C, L.e_pitch)) != DB_OK) return st;
+    if ((st = make_operand_map(&ga.e_lo, e_lo, rows_p, C, L.e_pitch)) != DB_OK) return st;
+
+    DB_CUDA_TRY(cudaMemsetAsync(base, 0, L.header_bytes, stream));
+
+    // 1. logits of every row, transposed orientation, split over D
+    {
+        tc::GemmArgs a{};
+        a.A = W; a.a_row = 1; a.a_k = C;          // A(m = class, k = feature) = W[k, m]
+        a.B = X; a.b_row = D; a.b_k = 1;          // B(n = sample, k = feature) = X[n, k]
+        a.out = partials; a.o_m = 1; a.o_n = C; a.o_split = rc;   // Z[n, m], one slab per split
+        a.M = C; a.N = static_cast<int>(rows); a.K = D; a.k_per_split = L.k_per_split; a.status = status;
+        st = launch_tc_gemm(a, L.n_tile, stream);
+        if (st != DB_OK) return st;
+    }
+    // 2. softmax residual with each worker's own 1/b, left split into TF32 halves beside the split X
+    {
+        SplitOut so{};
+        so.e_hi = e_hi; so.e_lo = e_lo; so.e_pitch = L.e_pitch;
+        so.X = X; so.x_hi = x_hi; so.x_lo = x_lo; so.x_pitch = L.x_pitch; so.D = D;
+        so.x_vec = (D % 4 == 0) && aligned16(X);
+        st = launch_softmax(partials, L.splits, rc, y, E, row_loss, rg, static_cast<int>(rows), C, tickets, losses,
+                            stream, true, &so);
+        if (st != DB_OK) return st;
+    }
+    // 3. one gradient per worker: G_w = X_w^T E_w, reduction over that worker's rows only
+    {
+        // largest batches first: their CTAs run longest and should not form the tail of the grid
+        int order[DB_MAX_K];
+        for (int w = 0; w < K; ++w) order[w] = w;
+        std::stable_sort(order, order + K, [&](int u, int v) {
+            return offsets[u + 1] - offsets[u] > offsets[v + 1] - offsets[v];
+        });
+        int max_steps = 1;
+        for (int z = 0; z < K; ++z) {
+            const int w = order[z];
+            ga.out[z] = G[w];
+            ga.row0[z] = rg.poff[w];
+            ga.steps[z] = (rg.poff[w + 1] - rg.poff[w]) / tcg::kStepRows;
+            max_steps = std::max(max_steps, ga.steps[z]);
+        }
+        ga.D = D; ga.C = C; ga.status = status;
+        // one main accumulator per four stages (chains of 16 additions), within the 512 columns
+        const int loads = (max_steps * tcg::kStepRows + tcg::kRowsPerStage - 1) / tcg::kRowsPerStage;
+        ga.n_acc = std::min(std::max((loads + 3) / 4, 1), tcg::kMaxAcc);
+        DB_CUDA_TRY(cudaFuncSetAttribute(tcg::grad_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         tcg::kSmemBytes));
+        dim3 grid((C + tcg::kTileN - 1) / tcg::kTileN, (D + tcg::kTileM - 1) / tcg::kTileM, K);
+        OverlappedLaunch OL(grid, dim3(tcg::kThreads), tcg::kSmemBytes, stream, true);
+        DB_CUDA_TRY(cudaLaunchKernelEx(&OL.cfg, tcg::grad_tma_kernel, ga));
+        DB_CUDA_TRY(cudaGetLastError());
+    }
+    return DB_OK;
 }
 
 }  // namespace
@@ -608,63 +746,8 @@ extern "C" db_status db_worker_grad_grouped(const float* X, const int32_t* y, co
     const long long rows = offsets[K];
     if (!valid_group_shape(rows, K, D, C)) return DB_ERR_ARG;
     if (reinterpret_cast<uintptr_t>(workspace) % 16) return DB_ERR_ARG;
-    const GroupedLayout L = grouped_layout(rows, K, D, C);
-    if (workspace_bytes < L.total()) return DB_ERR_ARG;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-
-    char* base = static_cast<char*>(workspace);
-    int* status = reinterpret_cast<int*>(base);
-    unsigned int* tickets = reinterpret_cast<unsigned int*>(base + kStatusBytes);
-    float* partials = reinterpret_cast<float*>(base + L.header_bytes);
-    float* E = reinterpret_cast<float*>(base + L.header_bytes + L.partial_bytes);
-    float* row_loss = reinterpret_cast<float*>(base + L.header_bytes + L.partial_bytes + L.e_bytes);
-    const long long rc = rows * C;
-    DB_CUDA_TRY(cudaMemsetAsync(base, 0, L.header_bytes, stream));
-
-    // 1. logits of every row, transposed orientation, split over D
-    {
-        tc::GemmArgs a{};
-        a.A = W; a.a_row = 1; a.a_k = C;
-        a.B = X; a.b_row = D; a.b_k = 1;
-        a.out = partials; a.o_m = 1; a.o_n = C; a.o_split = rc;
-        a.M = C; a.N = static_cast<int>(rows); a.K = D; a.k_per_split = L.k_per_split; a.status = status;
-        const db_status st = launch_tc_gemm(a, L.n_tile, stream);
-        if (st != DB_OK) return st;
-    }
-    // 2. softmax residual with each worker's own 1/b
-    RowGroups rg{};
-    rg.K = K;
-    for (int w = 0; w <= K; ++w) rg.off[w] = offsets[w];
-    {
-        const db_status st = launch_softmax(partials, L.splits, rc, y, E, row_loss, rg, static_cast<int>(rows), C,
-                                            tickets, losses, stream, true);
-        if (st != DB_OK) return st;
-    }
-    // 3. one gradient per worker: G_w = X_w^T E_w, reduction over that worker's rows only
-    {
-        tc::GemmArgs a{};
-        a.a_row = 1; a.a_k = D;
-        a.b_row = 1; a.b_k = C;
-        a.o_m = C; a.o_n = 1; a.o_split = 0;
-        a.M = D; a.N = C; a.status = status;
-        tc::GroupArgs gr{};
-        // largest batches first: their CTAs run longest and should not form the tail of the grid
-        int order[DB_MAX_K];
-        for (int w = 0; w < K; ++w) order[w] = w;
-        std::stable_sort(order, order + K, [&](int u, int v) {
-            return offsets[u + 1] - offsets[u] > offsets[v + 1] - offsets[v];
-        });
-        for (int z = 0; z < K; ++z) {
-            const int w = order[z];
-            gr.A[z] = X + static_cast<long long>(offsets[w]) * D;
-            gr.B[z] = E + static_cast<long long>(offsets[w]) * C;
-            gr.out[z] = G[w];
-            gr.K[z] = offsets[w + 1] - offsets[w];
-        }
-        const db_status st = launch_tc_gemm(a, 64, stream, &gr, K, true);
-        if (st != DB_OK) return st;
-    }
-    return DB_OK;
+    if (workspace_bytes < grouped_layout(rows, K, D, C).total()) return DB_ERR_ARG;
+    return worker_grad_tensor(X, y, W, offsets, K, D, C, G, losses, workspace, static_cast<cudaStream_t>(cuda_stream));
 }
 
 extern "C" db_status db_worker_grad(const float* X, const int32_t* y, const float* W, int32_t b_i,
