@@ -384,12 +384,12 @@ def measure_softmax(args, dev, rank, world):
         "config": {"workload": "softmax_D2048_C1000_b24_40_64_128", "D": D, "C": C, "batch_sizes": bs,
                    "l2": "L2 flushed (252 MB written, then read) before every timed step",
                    "calls": "db_worker_grad_grouped + db_aggregate_update_ex"},
-        "gpu_launches": 4 * steps, "clocks": sampler.summary(),
+        "gpu_launches": 5 * steps, "clocks": sampler.summary(),   # logits, softmax, gradients, aggregation, norm fold
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak, "peak_source": kind,
                      "note": "algorithmic FLOPs 4*sum(b)*D*C per step; the step is launch- and latency-bound "
                              "(reduction depth b_i <= 128), the tensor pipe is idle most of the time",
-                     "kernel": "tf32x3_gemm_kernel / tf32x3_gemm_grouped_kernel", "kernel_ms": ms,
+                     "kernel": "tf32x3_gemm_kernel (logits) / grad_tma_kernel (gradients)", "kernel_ms": ms,
                      "kernel_ms_min": float(np.min(per_step_ms)), "traffic": None},
     }
 

@@ -6,7 +6,7 @@
 // tc_gemm.cuh has to do; what is left of the operand preparation, the split of every fp32 value
 // into two TF32 halves, is done once by the kernel that produces E (and copies X), not once per
 // output tile.  A CTA of this kernel therefore only
-//   - copies [32 rows x 32 columns] boxes of the four split arrays (X_hi, X_lo, E_hi, E_lo) into
+//   - copies [16 rows x 32 columns] boxes of the four split arrays (X_hi, X_lo, E_hi, E_lo) into
 //     shared memory with cp.async.bulk.tensor (128-byte swizzle of 32-byte pieces, completion on an
 //     mbarrier),
 //   - issues three tcgen05.mma.kind::tf32 per 8 rows (lo*hi + hi*lo into one accumulator in tensor
@@ -17,7 +17,8 @@
 //
 // 192 threads: warp 0 (one lane) issues the TMA copies, warp 1 owns the tensor-memory allocation
 // and (one lane) issues the products, warps 2-5 are the epilogue.  Two shared-memory stages of
-// 48 KB, so two CTAs fit on an SM and one's epilogue overlaps the other's loads.  Every wait is
+// 24 KB (16 samples each), so four CTAs fit on an SM and their phases (copy, products, epilogue)
+// overlap; measured, a CTA's own phases are latency-bound and more resident CTAs pay.  Every wait is
 // bounded (see tc_gemm.cuh); on a time-out the copy thread waits, again bounded, for the copies it
 // has in flight before the CTA returns.
 #pragma once
@@ -32,9 +33,10 @@ constexpr int kTileM = 128;            // features per CTA = tensor-memory lanes
 constexpr int kTileN = 64;             // classes per CTA = accumulator columns
 constexpr int kChunk = 32;             // fp32 per 128-byte swizzled row
 constexpr int kStepRows = 8;           // reduction depth of one TF32 product
-constexpr int kRowsPerStage = 32;      // samples per stage: four products' worth
+constexpr int kRowsPerStage = 16;      // samples per stage: two products' worth
+constexpr int kAccRows = 32;           // consecutive samples whose hi*hi products share an accumulator turn
 constexpr int kStages = 2;
-constexpr int kChunkBytes = kRowsPerStage * 128;            // one [32 x 32] box
+constexpr int kChunkBytes = kRowsPerStage * 128;            // one [16 x 32] box
 constexpr int kAChunks = kTileM / kChunk, kBChunks = kTileN / kChunk;
 constexpr int kABytes = kAChunks * kChunkBytes;             // X_hi (or X_lo) part of a stage
 constexpr int kBBytes = kBChunks * kChunkBytes;             // E_hi (or E_lo) part of a stage
@@ -48,7 +50,7 @@ constexpr int kStagePitch = kTileN + 4;                     // floats per row of
 static_assert(kTileM * kStagePitch * 4 <= kStages * kStageBytes, "output staging fits in the operand stages");
 
 struct GradArgs {
-    CUtensorMap x_hi, x_lo;        // [padded rows, D], boxes of 32 x 32, 128-byte swizzle of 32-byte pieces
+    CUtensorMap x_hi, x_lo;        // [padded rows, D], boxes of 16 rows x 32, 128-byte swizzle of 32-byte pieces
     CUtensorMap e_hi, e_lo;        // [padded rows, C]
     float* out[DB_MAX_K];          // G_w, [D, C] row-major
     int row0[DB_MAX_K];            // first row of worker w in the split arrays (multiple of 8)
@@ -174,7 +176,9 @@ grad_tma_kernel(const __grid_constant__ GradArgs g) {
                 if (!alive) break;
                 tc::tc_fence_after();
                 const uint32_t st = tc::smem_u32(tiles + s * kStageBytes);
-                const uint32_t acc_main = tmem_base + (l % g.n_acc) * kTileN;
+                const int blk = l * kRowsPerStage / kAccRows;          // which 32-sample block
+                const bool blk_start = (l * kRowsPerStage) % kAccRows == 0;
+                const uint32_t acc_main = tmem_base + (blk % g.n_acc) * kTileN;
                 const int here = min(kRowsPerStage / kStepRows, steps - l * (kRowsPerStage / kStepRows));
                 for (int q = 0; q < here; ++q) {
                     const uint32_t off = q * 1024;      // 8 rows of 128 bytes
@@ -184,7 +188,7 @@ grad_tma_kernel(const __grid_constant__ GradArgs g) {
                     const uint64_t b_lo = smem_desc_mn_sw128(st + 2 * kABytes + kBBytes + off);
                     tc::mma_tf32(acc_cross, a_lo, b_hi, idesc, (l | q) != 0);
                     tc::mma_tf32(acc_cross, a_hi, b_lo, idesc, 1);
-                    tc::mma_tf32(acc_main, a_hi, b_hi, idesc, (l >= g.n_acc) || q != 0);
+                    tc::mma_tf32(acc_main, a_hi, b_hi, idesc, blk >= g.n_acc || !blk_start || q != 0);
                 }
                 tc::mma_commit(&empty_bar[s]);
             }
@@ -203,7 +207,7 @@ grad_tma_kernel(const __grid_constant__ GradArgs g) {
         const int quarter = warp & 3;                // the tensor-memory lanes this warp may read
         if (alive) {
             const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-            const int used = min(g.n_acc, loads);
+            const int used = min(g.n_acc, (steps * kStepRows + kAccRows - 1) / kAccRows);
             float* srow = reinterpret_cast<float*>(tiles) + (quarter * 32 + lane) * kStagePitch;
 #pragma unroll 1
             for (int c0 = 0; c0 < kTileN; c0 += 32) {

@@ -614,7 +614,7 @@ EncodeTiledFn encode_tiled() {
 }
 
 // Tensor map of a row-major fp32 array [rows, cols] with `pitch` floats per row, read in boxes of
-// 32 rows x 32 columns with the 128-byte swizzle of 32-byte pieces (the only one the tensor core takes
+// 16 rows x 32 columns with the 128-byte swizzle of 32-byte pieces (the only one the tensor core takes
 // for 32-bit operands that are contiguous along the output index); elements outside [rows, cols] read as zero.
 db_status make_operand_map(CUtensorMap* map, float* base, long long rows, long long cols, long long pitch) {
     EncodeTiledFn enc = encode_tiled();
@@ -707,9 +707,9 @@ db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, c
             max_steps = std::max(max_steps, ga.steps[z]);
         }
         ga.D = D; ga.C = C; ga.status = status;
-        // one main accumulator per four stages (chains of 16 additions), within the 512 columns
-        const int loads = (max_steps * tcg::kStepRows + tcg::kRowsPerStage - 1) / tcg::kRowsPerStage;
-        ga.n_acc = std::min(std::max((loads + 3) / 4, 1), tcg::kMaxAcc);
+        // one main accumulator per four 32-sample blocks (chains of 16 additions), within the 512 columns
+        const int blocks = (max_steps * tcg::kStepRows + tcg::kAccRows - 1) / tcg::kAccRows;
+        ga.n_acc = std::min(std::max((blocks + 3) / 4, 1), tcg::kMaxAcc);
         DB_CUDA_TRY(cudaFuncSetAttribute(tcg::grad_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          tcg::kSmemBytes));
         dim3 grid((C + tcg::kTileN - 1) / tcg::kTileN, (D + tcg::kTileM - 1) / tcg::kTileM, K);

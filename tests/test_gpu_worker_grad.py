@@ -129,6 +129,35 @@ def test_grouped_matches_the_oracle_per_worker(bs, D, C):
         assert abs(losses[w] - rloss) <= FP32_TOL * abs(rloss)
 
 
+@pytest.mark.parametrize("bs,D,C", [
+    ([1000, 3], 40, 72),                                   # 32 blocks of 32 samples: all seven main accumulators
+    ([4096], 64, 36),                                      # the longest reduction the tensor-core path takes
+    ([(7 * w) % 23 + 1 for w in range(64)], 130, 37),      # the maximum worker count; C % 4 != 0: element-wise stores
+    ([385, 384], 129, 65),                                 # 13 and 12 blocks: four accumulators, ragged tiles
+])
+def test_grouped_long_reductions_and_many_workers(bs, D, C):
+    X, y, W = inputs.softmax_problem(bs, D, C, seed=4100 + len(bs), w_std=0.05, device=DEV)
+    G, losses, offs = _grouped(X, y, W, bs)
+    Xh, yh, Wh = X.cpu().numpy(), y.cpu().numpy(), W.cpu().numpy()
+    for w in range(len(bs)):
+        rG, rloss = oracle.worker_grad(Xh[offs[w]:offs[w + 1]], yh[offs[w]:offs[w + 1]], Wh)
+        assert rel_err(f64(G[w]), rG) <= FP32_TOL, f"worker {w}"
+        assert abs(losses[w] - rloss) <= FP32_TOL * abs(rloss)
+
+
+def test_grouped_keeps_a_workers_nan_in_that_workers_gradient():
+    # worker 1's rows follow worker 0's in memory and share its last 16-sample copy; they must not leak
+    bs = [5, 9, 3]
+    X, y, W = inputs.softmax_problem(bs, 48, 20, seed=4200, w_std=0.05, device=DEV)
+    X[5:14] = float("nan")
+    G, _, offs = _grouped(X, y, W, bs)
+    Xh, yh, Wh = X.cpu().numpy(), y.cpu().numpy(), W.cpu().numpy()
+    for w in (0, 2):
+        rG, _ = oracle.worker_grad(Xh[offs[w]:offs[w + 1]], yh[offs[w]:offs[w + 1]], Wh)
+        assert rel_err(f64(G[w]), rG) <= FP32_TOL
+    assert bool(torch.isnan(G[1]).all())
+
+
 def test_grouped_then_aggregate_is_the_concatenated_batch_gradient():
     bs = [24, 40, 64, 128]
     D, C = 2048, 1000
