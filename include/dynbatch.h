@@ -284,7 +284,8 @@ db_status db_aggregate_update_host(db_host_pipeline* pipeline,
  *
  * On the tensor cores every fp32 product is formed from three TF32 products
  * (operands split into two TF32 halves, fp32 accumulation), which keeps the
- * result within 1e-5 of an fp64 evaluation.
+ * result within 1e-5 of an fp64 evaluation.  The tensor-core path is the grouped
+ * call below with one worker.
  * db_worker_grad is db_worker_grad_ex with flags = 0.
  * ------------------------------------------------------------------------ */
 #define DB_WORKER_GRAD_FFMA 1u
@@ -307,7 +308,10 @@ size_t db_worker_grad_workspace_bytes(int32_t b_i, int32_t D, int32_t C);
  *
  * The workers of one iteration share W, so their logits are one contraction
  * over the concatenated mini-batches; only the 1/b_w scale and the final
- * reduction over each worker's own rows differ.  Worker w owns rows
+ * reduction over each worker's own rows differ.  The last launch computes all
+ * K gradients; its operands (the softmax residual and X, split into TF32
+ * halves, every worker's rows padded with zero rows to a multiple of 8) reach
+ * the tensor cores by TMA.  Worker w owns rows
  * [offsets[w], offsets[w+1]) of X and y (its b_w = their number, Eq. 2's b_k)
  * and receives G[w] = X_w^T (softmax(X_w W) - Y_w) / b_w and losses[w].
  *
@@ -324,7 +328,8 @@ size_t db_worker_grad_workspace_bytes(int32_t b_i, int32_t D, int32_t C);
  *            offsets[K], K, D, C) bytes, 16-byte aligned, uninitialised; its
  *            first word is the status word described for db_worker_grad_ex
  * Tensor-core path only; results equal db_worker_grad's on each worker to
- * within the fp32 rounding of a differently split reduction over D.
+ * within the fp32 rounding of a differently split reduction over D.  NaN/Inf
+ * in one worker's samples stay in that worker's gradient and loss.
  * ------------------------------------------------------------------------ */
 db_status db_worker_grad_grouped(const float* X, const int32_t* y,
                                  const float* W, const int32_t* offsets,
