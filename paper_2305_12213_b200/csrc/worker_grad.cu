@@ -22,6 +22,7 @@
 #include "common.h"
 #include "tc_gemm.cuh"
 #include "tc_grad.cuh"
+#include "tc_logits.cuh"
 
 namespace dynbatch {
 namespace {
@@ -614,9 +615,11 @@ EncodeTiledFn encode_tiled() {
 }
 
 // Tensor map of a row-major fp32 array [rows, cols] with `pitch` floats per row, read in boxes of
-// 16 rows x 32 columns with the 128-byte swizzle of 32-byte pieces (the only one the tensor core takes
-// for 32-bit operands that are contiguous along the output index); elements outside [rows, cols] read as zero.
-db_status make_operand_map(CUtensorMap* map, float* base, long long rows, long long cols, long long pitch) {
+// box_rows rows x 32 columns; elements outside [rows, cols] read as zero.  Operands that are contiguous
+// along the output index need the 128-byte swizzle of 32-byte pieces (the only one the tensor core takes
+// for 32-bit operands in that orientation), operands contiguous along the reduction the ordinary one.
+db_status make_operand_map(CUtensorMap* map, const float* base, long long rows, long long cols, long long pitch,
+                           int box_rows, bool output_index_major) {
     EncodeTiledFn enc = encode_tiled();
     if (!enc) {
         record_message("cuTensorMapEncodeTiled is not available from this driver");
@@ -624,15 +627,45 @@ db_status make_operand_map(CUtensorMap* map, float* base, long long rows, long l
     }
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
     const cuuint64_t strides[1] = {static_cast<cuuint64_t>(pitch) * sizeof(float)};
-    const cuuint32_t box[2] = {tcg::kChunk, tcg::kRowsPerStage};
+    const cuuint32_t box[2] = {32, static_cast<cuuint32_t>(box_rows)};
     const cuuint32_t elem[2] = {1, 1};
-    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, elem,
-                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B,
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, elem,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           output_index_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
-        record_message("cuTensorMapEncodeTiled rejected the operand layout of the gradient contraction");
+        record_message("cuTensorMapEncodeTiled rejected an operand layout of the worker gradient");
         return DB_ERR_CUDA;
     }
+    return DB_OK;
+}
+
+// The logits with both operands copied by TMA from where the caller left them; needs 16-byte aligned
+// W and X and row pitches (C, D) that are multiples of 4 floats.
+db_status launch_logits_tma(const float* X, const float* W, float* partials, long long o_split, int rows, int D, int C,
+                            int k_per_split, int n_tile, int* status, cudaStream_t stream) {
+    tcl::LogitArgs a{};
+    db_status st;
+    if ((st = make_operand_map(&a.w, W, D, C, C, tcl::kBlockK, true)) != DB_OK) return st;
+    if ((st = make_operand_map(&a.x, X, rows, D, D, n_tile, false)) != DB_OK) return st;
+    a.out = partials; a.o_split = o_split; a.rows = rows; a.D = D; a.C = C; a.k_per_split = k_per_split;
+    a.status = status;
+    // one main accumulator per four reduction blocks (chains of 16 additions), within 512 columns
+    const int blocks = k_per_split / tcl::kBlockK;
+    a.n_acc = std::min(std::max((blocks + 3) / 4, 1), 512 / n_tile - 1);
+    const int splits = (D + k_per_split - 1) / k_per_split;
+    dim3 grid((rows + n_tile - 1) / n_tile, (C + tcl::kTileM - 1) / tcl::kTileM, splits);
+    void (*fn)(const tcl::LogitArgs) = nullptr;
+    int smem = 0;
+    switch (n_tile) {
+        case 32: fn = tcl::logits_tma_kernel<32>; smem = tcl::Smem<32>::kBytes; break;
+        case 64: fn = tcl::logits_tma_kernel<64>; smem = tcl::Smem<64>::kBytes; break;
+        default: fn = tcl::logits_tma_kernel<128>; smem = tcl::Smem<128>::kBytes; break;
+    }
+    DB_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    OverlappedLaunch OL(grid, dim3(tcl::kThreads), smem, stream, false);
+    DB_CUDA_TRY(cudaLaunchKernelEx(&OL.cfg, fn, a));
+    DB_CUDA_TRY(cudaGetLastError());
     return DB_OK;
 }
 
@@ -663,15 +696,20 @@ db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, c
 
     tcg::GradArgs ga{};
     db_status st;
-    if ((st = make_operand_map(&ga.x_hi, x_hi, rows_p, D, L.x_pitch)) != DB_OK) return st;
-    if ((st = make_operand_map(&ga.x_lo, x_lo, rows_p, D, L.x_pitch)) != DB_OK) return st;
-    if ((st = make_operand_map(&ga.e_hi, e_hi, rows_p, C, L.e_pitch)) != DB_OK) return st;
-    if ((st = make_operand_map(&ga.e_lo, e_lo, rows_p, C, L.e_pitch)) != DB_OK) return st;
+    if ((st = make_operand_map(&ga.x_hi, x_hi, rows_p, D, L.x_pitch, tcg::kRowsPerStage, true)) != DB_OK) return st;
+    if ((st = make_operand_map(&ga.x_lo, x_lo, rows_p, D, L.x_pitch, tcg::kRowsPerStage, true)) != DB_OK) return st;
+    if ((st = make_operand_map(&ga.e_hi, e_hi, rows_p, C, L.e_pitch, tcg::kRowsPerStage, true)) != DB_OK) return st;
+    if ((st = make_operand_map(&ga.e_lo, e_lo, rows_p, C, L.e_pitch, tcg::kRowsPerStage, true)) != DB_OK) return st;
 
     DB_CUDA_TRY(cudaMemsetAsync(base, 0, L.header_bytes, stream));
 
-    // 1. logits of every row, transposed orientation, split over D
-    {
+    // 1. logits of every row, transposed orientation, split over D; operands by TMA where their
+    //    alignment allows it, else through the register-converting contraction
+    if (aligned16(W) && aligned16(X) && C % 4 == 0 && D % 4 == 0) {
+        st = launch_logits_tma(X, W, partials, rc, static_cast<int>(rows), D, C, L.k_per_split, L.n_tile, status,
+                               stream);
+        if (st != DB_OK) return st;
+    } else {
         tc::GemmArgs a{};
         a.A = W; a.a_row = 1; a.a_k = C;          // A(m = class, k = feature) = W[k, m]
         a.B = X; a.b_row = D; a.b_k = 1;          // B(n = sample, k = feature) = X[n, k]
