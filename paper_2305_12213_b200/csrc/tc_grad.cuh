@@ -15,7 +15,7 @@
 // In the split arrays every worker's rows start at a multiple of 8 and are padded with zero rows to
 // a multiple of 8, the reduction depth of one TF32 product.
 //
-// 192 threads: warp 0 issues the TMA copies (12 lanes, one box each), warp 1 owns the tensor-memory allocation
+// 192 threads: warp 0 (one lane) issues the TMA copies, warp 1 owns the tensor-memory allocation
 // and (one lane) issues the products, warps 2-5 are the epilogue.  Two shared-memory stages of
 // 24 KB (16 samples each), so four CTAs fit on an SM and their phases (copy, products, epilogue)
 // overlap; measured, a CTA's own phases are latency-bound and more resident CTAs pay.  Every wait is
@@ -132,36 +132,30 @@ grad_tma_kernel(const __grid_constant__ GradArgs g) {
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA copies
-        // A stage is 12 boxes: 4 column chunks of X_hi and of X_lo, 2 of E_hi and of E_lo.  Lane i issues
-        // box i, all in the same instruction: one thread gets only about 2.5 million copies per second
-        // through (measured), while 8 lanes issuing together take barely longer than one.
-        constexpr int kBoxes = 2 * kAChunks + 2 * kBChunks;
-        const bool is_x = lane < 2 * kAChunks;
-        const int sub = is_x ? lane : lane - 2 * kAChunks;               // hi chunks first, then lo chunks
-        const int per = is_x ? kAChunks : kBChunks;
-        const bool is_lo = sub >= per;
-        const int chunk = sub - (is_lo ? per : 0);
-        const CUtensorMap* map = is_x ? (is_lo ? &g.x_lo : &g.x_hi) : (is_lo ? &g.e_lo : &g.e_hi);
-        const uint32_t box_off = (is_x ? 0 : 2 * kABytes) + (is_lo ? (is_x ? kABytes : kBBytes) : 0) + chunk * kChunkBytes;
-        const int col = (is_x ? m0 : n0) + chunk * kChunk;
-        int issued = 0;
-        for (int l = 0; l < loads; ++l) {
-            const int s = l % kStages;
-            int ok = 1;
-            if (lane == 0) {
-                if (l >= kStages) ok = tc::mbar_wait(&empty_bar[s], ((l / kStages) - 1) & 1, &abort_flag, g.status, 4);
-                if (abort_flag) ok = 0;
-                if (ok) mbar_expect_tx(&full_bar[s], kStageBytes);
-            }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok) break;
-            if (lane < kBoxes)
-                tma_load_2d(tc::smem_u32(tiles + s * kStageBytes) + box_off, map, col, g.row0[z] + l * kRowsPerStage,
-                            &full_bar[s]);
-            __syncwarp();
-            issued = l + 1;
-        }
         if (lane == 0) {
+            int issued = 0;
+            for (int l = 0; l < loads; ++l) {
+                const int s = l % kStages;
+                if (l >= kStages &&
+                    !tc::mbar_wait(&empty_bar[s], ((l / kStages) - 1) & 1, &abort_flag, g.status, 4))
+                    break;
+                if (abort_flag) break;
+                mbar_expect_tx(&full_bar[s], kStageBytes);
+                const uint32_t dst = tc::smem_u32(tiles + s * kStageBytes);
+                const int row = g.row0[z] + l * kRowsPerStage;
+#pragma unroll
+                for (int c = 0; c < kAChunks; ++c) {
+                    tma_load_2d(dst + c * kChunkBytes, &g.x_hi, m0 + c * kChunk, row, &full_bar[s]);
+                    tma_load_2d(dst + kABytes + c * kChunkBytes, &g.x_lo, m0 + c * kChunk, row, &full_bar[s]);
+                }
+#pragma unroll
+                for (int c = 0; c < kBChunks; ++c) {
+                    tma_load_2d(dst + 2 * kABytes + c * kChunkBytes, &g.e_hi, n0 + c * kChunk, row, &full_bar[s]);
+                    tma_load_2d(dst + 2 * kABytes + kBBytes + c * kChunkBytes, &g.e_lo, n0 + c * kChunk, row,
+                                &full_bar[s]);
+                }
+                issued = l + 1;
+            }
             // the copies issued last write into this CTA's shared memory until they land: see them
             // complete (bounded) before this thread lets the CTA exit, whatever the other roles do
             for (int l = max(0, issued - kStages); l < issued; ++l) {
