@@ -389,7 +389,7 @@ def measure_softmax(args, dev, rank, world):
                      "frac": achieved / peak, "peak_source": kind,
                      "note": "algorithmic FLOPs 4*sum(b)*D*C per step; the step is launch- and latency-bound "
                              "(reduction depth b_i <= 128), the tensor pipe is idle most of the time",
-                     "kernel": "tf32x3_gemm_kernel (logits) / grad_tma_kernel (gradients)", "kernel_ms": ms,
+                     "kernel": "logits_tma_kernel (logits) / grad_tma_kernel (gradients)", "kernel_ms": ms,
                      "kernel_ms_min": float(np.min(per_step_ms)), "traffic": None},
     }
 

@@ -11,11 +11,11 @@
 //      the last CTA of a worker also folds the per-sample losses into the mean;
 //   3. gradient: G = X^T E, reduction depth b_i.
 // The two contractions run on the tensor cores (tcgen05, three TF32 products per
-// fp32 product).  The logits use the general contraction of tc_gemm.cuh, which
-// converts fp32 operands on the fly; for the gradient the softmax kernel leaves E
-// and a copy of X already split into TF32 halves, row-major, and the contraction of
-// tc_grad.cuh reads them with TMA.  An fp32 FFMA version on shared-memory tiles is
-// kept as the accuracy reference and for very large b_i.
+// fp32 product), fed by TMA: the logits read W and X where the caller left them
+// (tc_logits.cuh; unaligned inputs go through the register-converting contraction of
+// tc_gemm.cuh), and for the gradient the softmax kernel leaves E and a copy of X
+// already split into TF32 halves, row-major (tc_grad.cuh).  An fp32 FFMA version on
+// shared-memory tiles is kept as the accuracy reference and for very large b_i.
 #include <algorithm>
 #include <cstdint>
 
