@@ -84,6 +84,7 @@ __device__ __forceinline__ void store_norm_partial(double* partials, double sq) 
 static __global__ void __launch_bounds__(1024) norm_finalize_kernel(const double* __restrict__ partials, long long n,
                                                              double* __restrict__ sq_out) {
     __shared__ double smem[32];
+    griddep_launch_dependents();     // the next step's kernel may be scheduled; it waits for this one itself
     griddep_wait();
     double acc = 0.0;
     for (long long i = threadIdx.x; i < n; i += blockDim.x) acc += __ldcg(partials + i);

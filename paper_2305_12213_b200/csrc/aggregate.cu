@@ -111,7 +111,11 @@ agg_vec_kernel(const __grid_constant__ AggArgs a) {
     constexpr int kQuads = kLanes / 4;
     const int K = KT > 0 ? KT : a.K;
     double sq = 0.0;
-    if (NORM) agg::griddep_launch_dependents();   // the norm's finalize kernel may be scheduled already
+    // Programmatic dependent launch, both ways: the kernel behind this one in the stream (the norm's fold, or
+    // the next step) may be scheduled already, and this one, if it was itself scheduled early, touches
+    // memory only once its predecessor has completed.  Both are no-ops for ordinary launches.
+    agg::griddep_launch_dependents();
+    agg::griddep_wait();
 
     const long long tile = static_cast<long long>(BLOCK) * UNROLL;
 #pragma unroll 1
@@ -203,7 +207,8 @@ template <typename GT, bool NORM, int OPT>
 __global__ void __launch_bounds__(kBlock)
 agg_scalar_kernel(const __grid_constant__ AggArgs a) {
     double sq = 0.0;
-    if (NORM) agg::griddep_launch_dependents();
+    agg::griddep_launch_dependents();
+    agg::griddep_wait();
     const long long step = static_cast<long long>(gridDim.x) * kBlock;
     for (long long j = static_cast<long long>(blockIdx.x) * kBlock + threadIdx.x; j < a.n; j += step)
         update_scalar<GT, NORM, OPT>(a, a.K, j, sq);
@@ -379,7 +384,20 @@ db_status aggregate_launch(AggArgs a, int opt, const void* const* grads, db_dtyp
     } else {
         grid = scalar_grid(fn, N);
     }
-    fn<<<grid, block, 0, stream>>>(a);
+    // A whole-array step may be scheduled while its predecessor in the stream (typically the previous
+    // step's norm fold) still runs; the kernel waits for it before its first access.  The chunks of the
+    // host pipeline are ordered by events across streams and take ordinary launches.
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1]{};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (chunk_partials || chunk_ctas) ? 0 : 1;
+    DB_CUDA_TRY(cudaLaunchKernelEx(&cfg, fn, a));
     DB_CUDA_TRY(cudaGetLastError());
     if (chunk_ctas) *chunk_ctas = grid;
     if (norm && !chunk_partials) DB_CUDA_TRY(agg::launch_norm_finalize(a.partials, grid, a.sq_out, stream, true));
