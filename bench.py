@@ -91,8 +91,8 @@ WORKLOADS = {"resnet50": resnet50_workload, "bert_base": bert_base_workload, "sm
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the aggregation kernel on the
 # resnet50 workload, from the ncu capture summarised under profiles/, with the digest of the kernel
 # sources (aggregate.cu, agg_device.cuh) the counters belong to.  Reported as null once the source has changed.
-NCU_TRAFFIC = {"workload": "resnet50_arena_N25557032_K8_fp32_gbatch256", "bytes_per_launch": 1201799168,
-               "kernel_source_sha256": "b7a04965583f5d2fc336e404c08d5566dfc971edc7938df91bd11e52d18a2f7b"}
+NCU_TRAFFIC = {"workload": "resnet50_arena_N25557032_K8_fp32_gbatch256", "bytes_per_launch": 1202312704,
+               "kernel_source_sha256": "896b73941fef77edddd1df2a1cbe721c689a72c93cabf6b0c7f6fd7ca0346c6b"}
 
 
 def step_bytes(K: int, N: int, grad_bytes: int) -> int:
@@ -251,7 +251,11 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
     assert np.isfinite(final_sq) and final_sq > 0 and bool(torch.isfinite(p[:1024]).all())
 
     peak, peak_kind = measured_peak()
-    kernel_ms = float(np.mean(per_step_ms))
+    # The dominant kernel's launch duration, from CUDA events on its stream.  Back-to-back mode: the timed
+    # region's time per step (aggregation kernel + the norm fold scheduled under it, so it slightly
+    # overstates the kernel); the per-call probe also pays an event pair per step and loses the overlap of
+    # consecutive steps, it is reported beside it.  Flushed mode: the event pair around each step.
+    kernel_ms = elapsed_ms / steps if flush is None else float(np.mean(per_step_ms))
     achieved = bytes_step / (kernel_ms * 1e-3) / 1e9
     gname = "float" if wl.grad_dtype == torch.float32 else "__nv_bfloat16"
     out = {
@@ -272,6 +276,7 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": f"of {peak_kind}",
                      "kernel": f"agg_vec_kernel<{gname}, K={K if K <= 16 else 0}, norm, momentum>", "kernel_ms": kernel_ms,
+                     "kernel_ms_probe_mean": float(np.mean(per_step_ms)),
                      "kernel_ms_min": float(np.min(per_step_ms)), "traffic": kernel_traffic(wl.name)},
     }
     if with_e2e:
