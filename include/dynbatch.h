@@ -138,9 +138,9 @@ db_status db_aggregate_adam_ex(const void* const* grads, db_dtype grad_dtype,
  *   sizes        host, T element counts >= 0
  *   params, momentum   host arrays of T device pointers (fp32, sizes[t] each)
  *   device_table device scratch of >= db_multi_plan_device_bytes(...) bytes,
- *                256-byte aligned; the plan keeps its tensor descriptors, the
- *                pointer table, one record per CTA and the norm's partial sums
- *                there until it is destroyed.  Must outlive the plan.
+ *                256-byte aligned; the plan keeps one record per CTA (the
+ *                pointers of its tile of one tensor) and the norm's partial
+ *                sums there until it is destroyed.  Must outlive the plan.
  *   cuda_stream  (create) the tables are uploaded on it and the call waits for
  *                the upload; (step) the launch stream
  * A tensor whose buffers are all 16-byte aligned takes 128-bit accesses,
