@@ -202,6 +202,39 @@ def test_on_a_side_stream():
     _assert_close(gpu, ref)
 
 
+def test_back_to_back_steps_between_foreign_kernels_without_synchronising():
+    """Steps are scheduled under their predecessor in the stream (programmatic dependent launch) and
+    wait for it themselves.  Seven steps, each right behind a torch kernel that writes that step's
+    gradients, alternately with and without the norm, nothing synchronised until the end: the state
+    must be what the oracle gets from the same gradients in the same order."""
+    N, K, steps = 2_000_003, 5, 7
+    b = [7, 1, 0, 30, 12]
+    base = [inputs.worker_gradients(K, N, 1e-3, 700 + 10 * it, device=DEV) for it in range(steps)]
+    work = [[torch.empty_like(t) for t in base[0]] for _ in range(2)]
+    p = inputs.normal(N, 0.02, 41, DEV)
+    v = inputs.normal(N, 0.01, 42, DEV)
+    rp, rv = f64(p), f64(v)
+    sq = torch.zeros(steps, dtype=torch.float64, device=DEV)
+    ws = _workspace(K, N)
+    torch.cuda.synchronize()
+    for it in range(steps):
+        g = work[it % 2]
+        for k in range(K):
+            torch.mul(base[it][k], 2.0, out=g[k])          # a foreign kernel produces this step's gradients
+        binding.aggregate_update(g, b, p, v, 0.05, 0.9, sq[it:it + 1] if it % 2 == 0 else None,
+                                 ws if it % 2 == 0 else None)
+    torch.cuda.synchronize()
+    ref_sq = []
+    for it in range(steps):
+        _, s = oracle.aggregate_update([host_grad(t) * np.float32(2.0) for t in base[it]], b, rp, rv,
+                                       float(np.float32(0.05)), float(np.float32(0.9)))
+        ref_sq.append(s)
+    assert rel_err(f64(p), rp) <= FP32_TOL and rel_err(f64(v), rv) <= FP32_TOL
+    got = sq.cpu().numpy()
+    for it in range(0, steps, 2):
+        assert abs(got[it] - ref_sq[it]) <= FP32_TOL * ref_sq[it]
+
+
 # ------------------------------------------------------------------ the named configurations
 def _iterate(K, N, dtype, g_std, b0, X_of_iter, kp, lr, mu, iters, seed, full_at, sample=1 << 18):
     """Controller step + aggregate/update per iteration with fresh gradients; the oracle is run
