@@ -95,6 +95,25 @@ NCU_TRAFFIC = {"workload": "resnet50_arena_N25557032_K8_fp32_gbatch256", "bytes_
                "kernel_source_sha256": "896b73941fef77edddd1df2a1cbe721c689a72c93cabf6b0c7f6fd7ca0346c6b"}
 
 
+NOMINAL_HBM_GBS = 8000.0   # NVIDIA's published HBM3e figure for B200 (not verifiable here): context beside the measured peak
+
+
+def copy_probe(dev, nbytes: int = 1 << 30, reps: int = 10) -> float:
+    """GB/s (read + write) of a plain device-to-device copy of 1 GiB, timed like the steps."""
+    src = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    dst = torch.empty_like(src)
+    src.zero_()
+    for _ in range(3):
+        dst.copy_(src)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        dst.copy_(src)
+    e1.record()
+    torch.cuda.synchronize()
+    return 2.0 * nbytes * reps / (e0.elapsed_time(e1) * 1e-3) / 1e9
+
+
 def step_bytes(K: int, N: int, grad_bytes: int) -> int:
     """Algorithmic HBM bytes of one step: K gradient reads + read and write of params and momentum."""
     return K * N * grad_bytes + 4 * N * 4
@@ -279,7 +298,11 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
                      "kernel_ms_probe_mean": float(np.mean(per_step_ms)),
                      "kernel_ms_min": float(np.min(per_step_ms)), "traffic": kernel_traffic(wl.name)},
     }
+    out["roofline"]["frac_of_nominal"] = achieved / NOMINAL_HBM_GBS
+    out["roofline"]["nominal_peak"] = NOMINAL_HBM_GBS
     if with_e2e:
+        # context only: this run's own device-to-device copy, the kind of measurement the peak file holds
+        out["roofline"]["copy_probe_gbs"] = copy_probe(dev)
         out["e2e"] = measure_e2e(wl, args, dev, grads, p, v, b)
     if with_cpu and rank == 0 and world == 1:
         out["cpu_baseline"] = cpu_baseline(wl, host_gradients(grads), b)
