@@ -11,7 +11,9 @@
 //     mbarrier),
 //   - issues three tcgen05.mma.kind::tf32 per 8 rows (lo*hi + hi*lo into one accumulator in tensor
 //     memory, hi*hi round-robin into up to seven others, see tc_gemm.cuh for why), and
-//   - drains the accumulators and writes its 128 x 64 tile of G.
+//   - drains the accumulators and writes its 128 x 64 tile of G: through shared memory in the box
+//     layout of a TMA store when G is 16-byte aligned with rows of a multiple of 16 bytes, else as
+//     whole rows with ordinary stores.
 // In the split arrays every worker's rows start at a multiple of 8 and are padded with zero rows to
 // a multiple of 8, the reduction depth of one TF32 product.
 //
@@ -48,11 +50,14 @@ constexpr int kThreads = 64 + kEpilogueThreads;
 constexpr int kMaxAcc = 512 / kTileN - 1;                   // main accumulators beside the cross-term one
 constexpr int kStagePitch = kTileN + 4;                     // floats per row of the output staging tile
 static_assert(kTileM * kStagePitch * 4 <= kStages * kStageBytes, "output staging fits in the operand stages");
+static_assert(kTileM * kTileN * 4 <= kStages * kStageBytes, "so does the tile in the TMA store's box layout");
 
 struct GradArgs {
     CUtensorMap x_hi, x_lo;        // [padded rows, D], boxes of 16 rows x 32, 128-byte swizzle of 32-byte pieces
     CUtensorMap e_hi, e_lo;        // [padded rows, C]
     float* out[DB_MAX_K];          // G_w, [D, C] row-major
+    int tma_store;                 // G_w are 16-byte aligned and C % 4 == 0: out_map[] is valid, tiles leave by TMA
+    CUtensorMap out_map[DB_MAX_K]; // G_w as [D, C], boxes of 128 rows x 32 columns, 128-byte swizzle
     int row0[DB_MAX_K];            // first row of worker w in the split arrays (multiple of 8)
     int steps[DB_MAX_K];           // its padded row count / 8
     int D, C;
@@ -71,6 +76,16 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(tc::smem_u32(bar)) : "memory");
 }
+
+// One box from shared memory to a 2-D tensor map (rows and columns outside the tensor are not written),
+// as part of the thread's current bulk group.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Until the bulk groups of this thread have finished READING shared memory.
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of an operand stored output-index-major.  For 32-bit elements the
 // tensor core accepts this orientation only with the 128-byte swizzle that permutes 32-byte pieces
@@ -208,7 +223,8 @@ grad_tma_kernel(const __grid_constant__ GradArgs g) {
         if (alive) {
             const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
             const int used = min(g.n_acc, (steps * kStepRows + kAccRows - 1) / kAccRows);
-            float* srow = reinterpret_cast<float*>(tiles) + (quarter * 32 + lane) * kStagePitch;
+            const int row = quarter * 32 + lane;
+            float* srow = reinterpret_cast<float*>(tiles) + row * kStagePitch;
 #pragma unroll 1
             for (int c0 = 0; c0 < kTileN; c0 += 32) {
                 uint32_t r[32], x[32];
@@ -220,15 +236,36 @@ grad_tma_kernel(const __grid_constant__ GradArgs g) {
                     for (int j = 0; j < 32; ++j)
                         r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(x[j]));
                 }
+                if (g.tma_store) {
+                    // the box layout of the store: [32-column half][128 rows][128 bytes], 16-byte pieces
+                    // permuted by the row's low three bits (which also keeps these stores conflict-free)
+                    unsigned char* box = tiles + (c0 / 32) * (kTileM * 128) + row * 128;
 #pragma unroll
-                for (int j = 0; j < 32; j += 4)
-                    *reinterpret_cast<float4*>(srow + c0 + j) =
-                        make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
-                                    __uint_as_float(r[j + 3]));
+                    for (int j = 0; j < 32; j += 4)
+                        *reinterpret_cast<float4*>(box + (((j >> 2) ^ (row & 7)) << 4)) =
+                            make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                                        __uint_as_float(r[j + 3]));
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4)
+                        *reinterpret_cast<float4*>(srow + c0 + j) =
+                            make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                                        __uint_as_float(r[j + 3]));
+                }
             }
+            if (g.tma_store) tc::fence_proxy_async_smem();    // the TMA engine reads what these threads wrote
         }
         asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
-        if (alive) {
+        if (alive && g.tma_store) {
+            if (et == 0) {
+#pragma unroll
+                for (int h = 0; h < kTileN / 32; ++h)
+                    if (n0 + h * 32 < g.C)
+                        tma_store_2d(&g.out_map[z], n0 + h * 32, m0, tc::smem_u32(tiles + h * (kTileM * 128)));
+                bulk_commit();
+                bulk_wait_read();      // shared memory must stay until the engine has read the tile
+            }
+        } else if (alive) {
             // whole rows of the tile, 16 threads per row
             const float* stage = reinterpret_cast<const float*>(tiles);
             float* obase = g.out[z];

@@ -745,6 +745,11 @@ db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, c
             max_steps = std::max(max_steps, ga.steps[z]);
         }
         ga.D = D; ga.C = C; ga.status = status;
+        // the tiles leave by TMA when every G_w allows it (16-byte aligned, rows a multiple of 16 bytes)
+        ga.tma_store = C % 4 == 0;
+        for (int z = 0; z < K && ga.tma_store; ++z) ga.tma_store = aligned16(ga.out[z]);
+        for (int z = 0; z < K && ga.tma_store; ++z)
+            if ((st = make_operand_map(&ga.out_map[z], ga.out[z], D, C, C, tcg::kTileM, false)) != DB_OK) return st;
         // one main accumulator per four 32-sample blocks (chains of 16 additions), within the 512 columns
         const int blocks = (max_steps * tcg::kStepRows + tcg::kAccRows - 1) / tcg::kAccRows;
         ga.n_acc = std::min(std::max((blocks + 3) / 4, 1), tcg::kMaxAcc);
