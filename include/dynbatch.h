@@ -350,7 +350,10 @@ size_t db_worker_grad_grouped_workspace_bytes(int32_t total_rows, int32_t K,
  *   A(m, k) = A[m * a_row + k * a_k],  B(n, k) = B[n * b_row + k * b_k]
  *   out(m, n) at out[m * o_m + n * o_n]       all device fp32, strides in
  *   elements, >= 0 (outputs >= 1); either operand may be contiguous along k or
- *   along its rows, which selects 128-bit loads when 16-byte aligned.
+ *   along its rows, which selects 128-bit loads when 16-byte aligned.  With A
+ *   contiguous along m, B along k and out along m (a_row = b_k = o_m = 1, bases
+ *   16-byte aligned, a_k and b_row multiples of 4) the operands travel by TMA,
+ *   as for the logits of db_worker_grad.
  *   M, N >= 1, K >= 0 (K = 0 writes zeros)
  *   status   device, one int32 the caller has cleared; set non-zero if a
  *            time-limited wait inside the kernel gave up

@@ -49,8 +49,8 @@ struct Smem {
 struct LogitArgs {
     CUtensorMap w;                 // [D, C] fp32, boxes of 32 rows x 32 columns, 128-byte swizzle of 32-byte pieces
     CUtensorMap x;                 // [rows, D] fp32, boxes of N_TILE rows x 32 columns, 128-byte swizzle
-    float* out;                    // Z(n, c) at out[split * o_split + n * C + c]
-    long long o_split;
+    float* out;                    // Z(n, c) at out[split * o_split + n * o_n + c]
+    long long o_split, o_n;
     int rows, D, C;
     int k_per_split;               // multiple of 32
     int n_acc;                     // main accumulators, (n_acc + 1) * N_TILE <= 512
@@ -267,12 +267,12 @@ logits_tma_kernel(const __grid_constant__ LogitArgs g) {
                 }
                 const int n_first = n0 + c0;
                 if (m >= g.C || n_first >= g.rows) continue;
-                float* col = obase + static_cast<long long>(n_first) * g.C;
+                float* col = obase + static_cast<long long>(n_first) * g.o_n;
                 const int n_left = g.rows - n_first;
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     if (j < n_left) *col = __uint_as_float(r[j]);
-                    col += g.C;
+                    col += g.o_n;
                 }
             }
         }

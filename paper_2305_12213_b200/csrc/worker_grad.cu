@@ -455,6 +455,9 @@ db_status launch_tc_gemm(tc::GemmArgs a, int n_tile, cudaStream_t stream, bool o
 bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
 
 // defined below, beside the grouped entry point
+db_status launch_logits_tma(const float* X, long long x_pitch, const float* W, long long w_pitch, float* partials,
+                            long long o_split, long long o_n, int rows, int D, int C, int k_per_split, int n_tile,
+                            int* status, cudaStream_t stream);
 size_t grouped_workspace_total(long long rows, int K, int D, int C);
 db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, const int32_t* offsets, int K, int D,
                              int C, float* const* G, float* losses, void* workspace, cudaStream_t stream);
@@ -472,14 +475,20 @@ extern "C" db_status db_contract_f32(const float* A, int64_t a_row, int64_t a_k,
     if (reinterpret_cast<uintptr_t>(A) % 4 || reinterpret_cast<uintptr_t>(B) % 4 ||
         reinterpret_cast<uintptr_t>(out) % 4 || reinterpret_cast<uintptr_t>(status) % 4)
         return DB_ERR_ARG;
+    const int n_tile = N <= 32 ? 32 : (N <= 64 ? 64 : 128);
+    const int k_round = K > 0 ? (K + tc::kBlockK - 1) / tc::kBlockK * tc::kBlockK : tc::kBlockK;
+    // A contiguous along m, B along k, out along m: the layout of the logits, operands by TMA
+    if (K > 0 && a_row == 1 && a_k % 4 == 0 && aligned16(A) && b_k == 1 && b_row % 4 == 0 && aligned16(B) && o_m == 1)
+        return launch_logits_tma(B, b_row, A, a_k, out, 0, o_n, N, K, M, k_round, n_tile, status,
+                                 static_cast<cudaStream_t>(cuda_stream));
     tc::GemmArgs a{};
     a.A = A; a.a_row = a_row; a.a_k = a_k;
     a.B = B; a.b_row = b_row; a.b_k = b_k;
     a.out = out; a.o_m = o_m; a.o_n = o_n; a.o_split = 0;
     a.M = M; a.N = N; a.K = K;
-    a.k_per_split = K > 0 ? (K + tc::kBlockK - 1) / tc::kBlockK * tc::kBlockK : tc::kBlockK;
+    a.k_per_split = k_round;
     a.status = status;
-    return launch_tc_gemm(a, N <= 32 ? 32 : (N <= 64 ? 64 : 128), static_cast<cudaStream_t>(cuda_stream));
+    return launch_tc_gemm(a, n_tile, static_cast<cudaStream_t>(cuda_stream));
 }
 
 extern "C" size_t db_worker_grad_workspace_bytes(int32_t b_i, int32_t D, int32_t C) {
@@ -640,14 +649,17 @@ db_status make_operand_map(CUtensorMap* map, const float* base, long long rows, 
     return DB_OK;
 }
 
-// The logits with both operands copied by TMA from where the caller left them; needs 16-byte aligned
-// W and X and row pitches (C, D) that are multiples of 4 floats.
-db_status launch_logits_tma(const float* X, const float* W, float* partials, long long o_split, int rows, int D, int C,
-                            int k_per_split, int n_tile, int* status, cudaStream_t stream) {
+// out(n, c) = sum_d X(n, d) W(d, c) with both operands copied by TMA from where the caller left them
+// (the logits; also db_contract_f32 for operands laid out that way).  Needs 16-byte aligned W and X and
+// row pitches that are multiples of 4 floats; out(n, c) lands at out[split * o_split + n * o_n + c].
+db_status launch_logits_tma(const float* X, long long x_pitch, const float* W, long long w_pitch, float* partials,
+                            long long o_split, long long o_n, int rows, int D, int C, int k_per_split, int n_tile,
+                            int* status, cudaStream_t stream) {
     tcl::LogitArgs a{};
     db_status st;
-    if ((st = make_operand_map(&a.w, W, D, C, C, tcl::kBlockK, true)) != DB_OK) return st;
-    if ((st = make_operand_map(&a.x, X, rows, D, D, n_tile, false)) != DB_OK) return st;
+    if ((st = make_operand_map(&a.w, W, D, C, w_pitch, tcl::kBlockK, true)) != DB_OK) return st;
+    if ((st = make_operand_map(&a.x, X, rows, D, x_pitch, n_tile, false)) != DB_OK) return st;
+    a.o_n = o_n;
     a.out = partials; a.o_split = o_split; a.rows = rows; a.D = D; a.C = C; a.k_per_split = k_per_split;
     a.status = status;
     // one main accumulator per four reduction blocks (chains of 16 additions), within 512 columns
@@ -706,8 +718,8 @@ db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, c
     // 1. logits of every row, transposed orientation, split over D; operands by TMA where their
     //    alignment allows it, else through the register-converting contraction
     if (aligned16(W) && aligned16(X) && C % 4 == 0 && D % 4 == 0) {
-        st = launch_logits_tma(X, W, partials, rc, static_cast<int>(rows), D, C, L.k_per_split, L.n_tile, status,
-                               stream);
+        st = launch_logits_tma(X, D, W, C, partials, rc, C, static_cast<int>(rows), D, C, L.k_per_split, L.n_tile,
+                               status, stream);
         if (st != DB_OK) return st;
     } else {
         tc::GemmArgs a{};

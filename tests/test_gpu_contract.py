@@ -34,6 +34,22 @@ def test_against_fp64_matmul(M, N, K, la, lb):
     assert rel_err(f64(out), ref) <= FP32_TOL
 
 
+@pytest.mark.parametrize("M,N,K", [(4, 1, 4), (128, 32, 32), (132, 33, 68), (300, 130, 100), (1000, 24, 128),
+                                   (260, 1000, 40), (1000, 256, 2048), (1000, 128, 4100)])
+def test_operands_by_tma_in_the_logits_layout(M, N, K):
+    """A contiguous along m, B along k, out along m (all 16-byte aligned, pitches multiples of 4): the
+    layout of the logits, which takes the TMA-fed kernel; ragged tiles, a ragged last reduction block,
+    reductions long enough for several accumulators."""
+    A, B = _operand(M, K, "row", 5), _operand(N, K, "k", 6)
+    out_t = torch.full((N, M), float("nan"), device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    binding.contract_f32(A, B, out_t.t(), status)          # out(m, n) stored at [n, m]
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref = f64(A) @ f64(B).T
+    assert rel_err(f64(out_t.t()), ref) <= FP32_TOL
+
+
 def test_empty_reduction_writes_zeros():
     import ctypes
     M, N = 70, 40
