@@ -216,10 +216,34 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
     if wl.working_set < 2 * L2_BYTES:
         flush = torch.empty(2 * L2_BYTES // 4, dtype=torch.int32, device=dev)
 
+    variant = getattr(args, "variant", "momentum")
+    state_bytes = 16                      # p and v read and written
+    kernel_label = "agg_vec_kernel"
+    adam_t = 0
+    if variant == "adam":
+        u = torch.zeros(N, device=dev)    # second moment; v serves as the first
+        state_bytes = 24
+    elif variant == "tensor_list":
+        if N not in (inputs.RESNET50_N, inputs.BERT_BASE_N):
+            raise SystemExit("--variant tensor_list needs a workload with a tensor list (resnet50, bert_base)")
+        # the same memory seen as the model's separately allocated tensors, one launch through a plan
+        shapes = inputs.resnet50_tensor_shapes() if N == inputs.RESNET50_N else inputs.bert_base_tensor_shapes()
+        offs = inputs.tensor_offsets(shapes)
+        assert offs[-1] == N
+        cut = lambda t: [t[s:e] for s, e in zip(offs[:-1], offs[1:])]
+        plan = binding.MultiTensorPlan([cut(g) for g in grads], cut(p), cut(v))
+        kernel_label = f"agg_multi_kernel over {len(shapes)} tensors"
+
     def step():
-        nonlocal b
+        nonlocal b, adam_t
         b = binding.controller_step(b, wl.throughputs, wl.kp)
-        binding.aggregate_update(grads, b, p, v, wl.lr, wl.mu, sq, ws, stream)
+        if variant == "adam":
+            adam_t += 1
+            binding.aggregate_adam(grads, b, p, v, u, 1e-3, 0.9, 0.999, 1e-8, adam_t, sq, ws, stream)
+        elif variant == "tensor_list":
+            plan.step(b, wl.lr, wl.mu, sq, stream)
+        else:
+            binding.aggregate_update(grads, b, p, v, wl.lr, wl.mu, sq, ws, stream)
 
     warmup = max(3, args.warmup)
     for _ in range(warmup):
@@ -264,7 +288,7 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
         per_step_ms = [e0.elapsed_time(e1) for e0, e1 in pairs]
         elapsed_ms = float(np.sum(per_step_ms))
     replicas.barrier(dev)
-    bytes_step = wl.bytes_per_step
+    bytes_step = wl.K * wl.N * wl.grad_bytes + state_bytes * wl.N
     job_bps, max_ms = replicas.job_throughput(bytes_step * steps, elapsed_ms, dev)
     final_sq = float(sq.item())
     assert np.isfinite(final_sq) and final_sq > 0 and bool(torch.isfinite(p[:1024]).all())
@@ -278,12 +302,13 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
     achieved = bytes_step / (kernel_ms * 1e-3) / 1e9
     gname = "float" if wl.grad_dtype == torch.float32 else "__nv_bfloat16"
     out = {
-        "metric": METRIC, "value": job_bps / 1e9, "unit": "GB/s",
+        "metric": METRIC if variant == "momentum" else f"{METRIC} [{variant} variant of the step]",
+        "value": job_bps / 1e9, "unit": "GB/s",
         "iterations_per_s": world * steps / (max_ms * 1e-3),
         "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": max_ms / steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": wl.name, "K": K, "N": N,
+        "config": {"workload": wl.name if variant == "momentum" else f"{wl.name}_{variant}", "K": K, "N": N,
                    "grad_dtype": "f32" if wl.grad_dtype == torch.float32 else "bf16",
                    "global_batch": sum(wl.b0), "kp": wl.kp, "lr": wl.lr, "mu": wl.mu, "grad_sqnorm": True,
                    "bytes_per_step": bytes_step,
@@ -294,12 +319,16 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
         "clocks": sampler.summary(),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": f"of {peak_kind}",
-                     "kernel": f"agg_vec_kernel<{gname}, K={K if K <= 16 else 0}, norm, momentum>", "kernel_ms": kernel_ms,
+                     "kernel": f"{kernel_label}<{gname}, K={K if K <= 16 else 0}, norm, {'adam' if variant == 'adam' else 'momentum'}>",
+                     "kernel_ms": kernel_ms,
                      "kernel_ms_probe_mean": float(np.mean(per_step_ms)),
-                     "kernel_ms_min": float(np.min(per_step_ms)), "traffic": kernel_traffic(wl.name)},
+                     "kernel_ms_min": float(np.min(per_step_ms)),
+                     "traffic": kernel_traffic(wl.name) if variant == "momentum" else None},
     }
     out["roofline"]["frac_of_nominal"] = achieved / NOMINAL_HBM_GBS
     out["roofline"]["nominal_peak"] = NOMINAL_HBM_GBS
+    if variant != "momentum":
+        return out                        # the end-to-end and CPU legs belong to the headline step
     if with_e2e:
         # context only: this run's own device-to-device copy, the kind of measurement the peak file holds
         out["roofline"]["copy_probe_gbs"] = copy_probe(dev)
@@ -537,6 +566,10 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--variant", choices=["momentum", "adam", "tensor_list"], default="momentum",
+                    help="the step's optimizer / entry point (resnet50 and bert_base workloads): momentum = "
+                         "db_aggregate_update_ex (headline), adam = db_aggregate_adam_ex, tensor_list = "
+                         "db_aggregate_update_multi over the model's separate tensors")
     ap.add_argument("--workload", choices=["resnet50", "bert_base", "small", "sweep", "softmax"], default="resnet50",
                     help="resnet50 is the headline configuration; sweep prints one line per (N, K) point")
     args = ap.parse_args()
