@@ -468,7 +468,13 @@ def run_ours(args):
         if rank == 0:
             print(json.dumps(out), flush=True)
     elif args.workload == "sweep":
-        for wl in sweep_workloads():
+        points = sweep_workloads()
+        if args.sweep_point:
+            n_sel, k_sel = (int(x) for x in args.sweep_point.split(","))
+            points = [w for w in points if w.N == n_sel and w.K == k_sel]
+            if not points:
+                raise SystemExit("--sweep-point: no such point (N in 2^20..2^28 by 4x, K in 2,4,8,16,32, K*N <= 2^33)")
+        for wl in points:
             out = measure(wl, args, dev, rank, world, with_e2e=False, with_cpu=False)
             if rank == 0:
                 print(json.dumps(out), flush=True)
@@ -570,6 +576,8 @@ def main():
                     help="the step's optimizer / entry point (resnet50 and bert_base workloads): momentum = "
                          "db_aggregate_update_ex (headline), adam = db_aggregate_adam_ex, tensor_list = "
                          "db_aggregate_update_multi over the model's separate tensors")
+    ap.add_argument("--sweep-point", default="", metavar="N,K",
+                    help="with --workload sweep: run only this point (e.g. 67108864,2), for profiler captures")
     ap.add_argument("--workload", choices=["resnet50", "bert_base", "small", "sweep", "softmax"], default="resnet50",
                     help="resnet50 is the headline configuration; sweep prints one line per (N, K) point")
     args = ap.parse_args()
