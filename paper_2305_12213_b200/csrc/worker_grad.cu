@@ -713,6 +713,27 @@ db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, c
     if ((st = make_operand_map(&ga.e_hi, e_hi, rows_p, C, L.e_pitch, tcg::kRowsPerStage, true)) != DB_OK) return st;
     if ((st = make_operand_map(&ga.e_lo, e_lo, rows_p, C, L.e_pitch, tcg::kRowsPerStage, true)) != DB_OK) return st;
 
+    // largest batches first: their CTAs run longest and should not form the tail of the grid
+    int order[DB_MAX_K];
+    for (int w = 0; w < K; ++w) order[w] = w;
+    std::stable_sort(order, order + K, [&](int u, int v) {
+        return offsets[u + 1] - offsets[u] > offsets[v + 1] - offsets[v];
+    });
+    int max_steps = 1;
+    for (int z = 0; z < K; ++z) {
+        const int w = order[z];
+        ga.out[z] = G[w];
+        ga.row0[z] = rg.poff[w];
+        ga.steps[z] = (rg.poff[w + 1] - rg.poff[w]) / tcg::kStepRows;
+        max_steps = std::max(max_steps, ga.steps[z]);
+    }
+    // the tiles leave by TMA when every G_w allows it (16-byte aligned, rows a multiple of 16 bytes)
+    ga.tma_store = C % 4 == 0;
+    for (int z = 0; z < K && ga.tma_store; ++z) ga.tma_store = aligned16(ga.out[z]);
+    for (int z = 0; z < K && ga.tma_store; ++z)
+        if ((st = make_operand_map(&ga.out_map[z], ga.out[z], D, C, C, tcg::kTileM, false)) != DB_OK) return st;
+
+    // nothing has been enqueued up to here
     DB_CUDA_TRY(cudaMemsetAsync(base, 0, L.header_bytes, stream));
 
     // 1. logits of every row, transposed orientation, split over D; operands by TMA where their
@@ -742,26 +763,7 @@ db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, c
     }
     // 3. one gradient per worker: G_w = X_w^T E_w, reduction over that worker's rows only
     {
-        // largest batches first: their CTAs run longest and should not form the tail of the grid
-        int order[DB_MAX_K];
-        for (int w = 0; w < K; ++w) order[w] = w;
-        std::stable_sort(order, order + K, [&](int u, int v) {
-            return offsets[u + 1] - offsets[u] > offsets[v + 1] - offsets[v];
-        });
-        int max_steps = 1;
-        for (int z = 0; z < K; ++z) {
-            const int w = order[z];
-            ga.out[z] = G[w];
-            ga.row0[z] = rg.poff[w];
-            ga.steps[z] = (rg.poff[w + 1] - rg.poff[w]) / tcg::kStepRows;
-            max_steps = std::max(max_steps, ga.steps[z]);
-        }
         ga.D = D; ga.C = C; ga.status = status;
-        // the tiles leave by TMA when every G_w allows it (16-byte aligned, rows a multiple of 16 bytes)
-        ga.tma_store = C % 4 == 0;
-        for (int z = 0; z < K && ga.tma_store; ++z) ga.tma_store = aligned16(ga.out[z]);
-        for (int z = 0; z < K && ga.tma_store; ++z)
-            if ((st = make_operand_map(&ga.out_map[z], ga.out[z], D, C, C, tcg::kTileM, false)) != DB_OK) return st;
         // one main accumulator per four 32-sample blocks (chains of 16 additions), within the 512 columns
         const int blocks = (max_steps * tcg::kStepRows + tcg::kAccRows - 1) / tcg::kAccRows;
         ga.n_acc = std::min(std::max((blocks + 3) / 4, 1), tcg::kMaxAcc);
