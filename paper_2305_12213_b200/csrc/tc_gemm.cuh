@@ -395,6 +395,7 @@ __device__ __forceinline__ void tf32x3_gemm_body(const GemmArgs& g, const int sp
         }
         // ------------------------------------------------------------ epilogue
         if (alive && nkb > 0) alive = mbar_wait(&done_bar, 0, &abort_flag, g.status, 3);
+        alive = __all_sync(0xffffffffu, alive);      // tcgen05.ld below is a warp-wide instruction
         tc_fence_after();
         if (alive) {
             // warp w may read tensor-memory lanes 32 (w mod 4) .. +31; the two warps that share a lane

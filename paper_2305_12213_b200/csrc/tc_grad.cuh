@@ -216,7 +216,8 @@ grad_tma_kernel(const __grid_constant__ GradArgs g) {
         }
     } else {
         // ------------------------------------------------------------ epilogue
-        const bool alive = tc::mbar_wait(&done_bar, 0, &abort_flag, g.status, 6);
+        // the verdict is made the same for the whole warp: tcgen05.ld below is a warp-wide instruction
+        const bool alive = __all_sync(0xffffffffu, tc::mbar_wait(&done_bar, 0, &abort_flag, g.status, 6));
         tc::tc_fence_after();
         const int et = tid - 64;                     // 0..127
         const int quarter = warp & 3;                // the tensor-memory lanes this warp may read

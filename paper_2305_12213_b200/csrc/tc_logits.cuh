@@ -210,7 +210,8 @@ logits_tma_kernel(const __grid_constant__ LogitArgs g) {
         bool alive = true;
         for (int kb = 0; kb < nkb; ++kb) {
             const int s = kb % kStages;
-            alive = tc::mbar_wait(&full_bar[s], (kb / kStages) & 1, &abort_flag, g.status, 8);
+            // the verdict is made the same for the whole warp: what follows has warp-wide operations
+            alive = __all_sync(0xffffffffu, tc::mbar_wait(&full_bar[s], (kb / kStages) & 1, &abort_flag, g.status, 8));
             if (!alive) break;
             unsigned char* st = ring + s * L::kStage;
             // element-wise, so neither swizzle matters: a lo tile mirrors its hi tile's layout
@@ -239,6 +240,7 @@ logits_tma_kernel(const __grid_constant__ LogitArgs g) {
             if (lane == 0) tc::mbar_arrive(&split_bar[s]);
         }
         if (alive && nkb > 0) alive = tc::mbar_wait(&done_bar, 0, &abort_flag, g.status, 3);
+        alive = __all_sync(0xffffffffu, alive);      // tcgen05.ld below is a warp-wide instruction
         tc::tc_fence_after();
         if (alive) {
             // warp w may read tensor-memory lanes 32 (w mod 4) .. +31; the two warps that share a lane
