@@ -145,6 +145,25 @@ def test_grouped_long_reductions_and_many_workers(bs, D, C):
         assert abs(losses[w] - rloss) <= FP32_TOL * abs(rloss)
 
 
+def test_grouped_outputs_off_the_16_byte_grid_take_ordinary_stores():
+    # C is a multiple of 4 but the gradient buffers start one float past a 16-byte boundary: no TMA store
+    bs, D, C = [9, 40], 160, 72
+    X, y, W = inputs.softmax_problem(bs, D, C, seed=4300, w_std=0.05, device=DEV)
+    offs = [0] + list(np.cumsum(bs))
+    raw = [torch.full((D * C + 1,), float("nan"), device=DEV) for _ in bs]
+    G = [r[1:].view(D, C) for r in raw]
+    ws = torch.empty(binding.worker_grad_grouped_workspace_bytes(offs[-1], len(bs), D, C), dtype=torch.uint8,
+                     device=DEV)
+    binding.worker_grad_grouped(X, y, W, offs, G, None, ws)
+    torch.cuda.synchronize()
+    assert binding.worker_grad_status(ws) == 0
+    Xh, yh, Wh = X.cpu().numpy(), y.cpu().numpy(), W.cpu().numpy()
+    for w in range(len(bs)):
+        rG, _ = oracle.worker_grad(Xh[offs[w]:offs[w + 1]], yh[offs[w]:offs[w + 1]], Wh)
+        assert rel_err(f64(G[w]), rG) <= FP32_TOL
+        assert bool(torch.isnan(raw[w][0]))                 # the element before the buffer is untouched
+
+
 def test_grouped_keeps_a_workers_nan_in_that_workers_gradient():
     # worker 1's rows follow worker 0's in memory and share its last 16-sample copy; they must not leak
     bs = [5, 9, 3]
