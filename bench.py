@@ -74,14 +74,15 @@ def small_workload():
                     [1.0, 2.0, 5.0], 0.5, 0.1, 0.9, 1.0)
 
 
-def sweep_workloads():
+def sweep_workloads(grad_dtype=torch.float32):
     out = []
+    tag = "fp32" if grad_dtype == torch.float32 else "bf16"
     for n in (1 << 20, 1 << 22, 1 << 24, 1 << 26, 1 << 28):
         for k in (2, 4, 8, 16, 32):
             if n * k <= (1 << 33):
                 b = inputs.batch_sizes_uniform(k, 8, 256, 5000 + k)
                 # throughputs proportional to b: the controller step runs and holds b fixed
-                out.append(Workload(f"sweep_N{n}_K{k}_fp32", k, n, torch.float32, b, [float(x) for x in b],
+                out.append(Workload(f"sweep_N{n}_K{k}_{tag}", k, n, grad_dtype, b, [float(x) for x in b],
                                     1.0, 0.1, 0.9, 1.0))
     return out
 
@@ -468,7 +469,7 @@ def run_ours(args):
         if rank == 0:
             print(json.dumps(out), flush=True)
     elif args.workload == "sweep":
-        points = sweep_workloads()
+        points = sweep_workloads(torch.bfloat16 if args.sweep_dtype == "bf16" else torch.float32)
         if args.sweep_point:
             n_sel, k_sel = (int(x) for x in args.sweep_point.split(","))
             points = [w for w in points if w.N == n_sel and w.K == k_sel]
@@ -576,6 +577,8 @@ def main():
                     help="the step's optimizer / entry point (resnet50 and bert_base workloads): momentum = "
                          "db_aggregate_update_ex (headline), adam = db_aggregate_adam_ex, tensor_list = "
                          "db_aggregate_update_multi over the model's separate tensors")
+    ap.add_argument("--sweep-dtype", choices=["fp32", "bf16"], default="fp32",
+                    help="gradient storage of the sweep's points (the named sweep configuration is fp32)")
     ap.add_argument("--sweep-point", default="", metavar="N,K",
                     help="with --workload sweep: run only this point (e.g. 67108864,2), for profiler captures")
     ap.add_argument("--workload", choices=["resnet50", "bert_base", "small", "sweep", "softmax"], default="resnet50",
