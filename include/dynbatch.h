@@ -431,7 +431,9 @@ db_status db_static_allocate(const double* throughputs, int32_t K, int32_t b0,
  *
  *   b0          host, K initial batch sizes >= 1
  *   kp          0 < kp <= 1;  alpha 0 < alpha <= 1;  dead_band >= 0
- *   b_min,b_max host, K each, or NULL for 1 and sum(b0)
+ *   b_min,b_max host, K each, or NULL for 1 and sum(b0); b_min[k] >= 1 (a
+ *               worker at batch 0 would have no iteration time to observe)
+ *               and b_max[k] >= b_min[k], else DB_ERR_ARG
  * db_controller_observe: b_out (host, K, nullable) receives the batch sizes in
  * force after the observation, *changed (nullable) whether they moved.
  * Not thread-safe per object.  All arithmetic is IEEE fp64 in a fixed order.

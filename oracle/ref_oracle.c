@@ -14,8 +14,8 @@
  *   - the static throughput-proportional allocation  (Section 3.2)
  *   - the mean cross-entropy gradient of a bias-free linear-softmax
  *     classifier, used to check the weighting against the gradient of the
- *     concatenated batch (Section 3.1: the weighted average "maintains
- *     equivalence with conventional uniform batching").
+ *     concatenated batch (Section 3.1: the weights sum to one, so equal
+ *     batches give the plain mean of Eq. 1).
  *
  * Only tests, the smoke check and the CPU-baseline timing may call this
  * file.  It shares no code, header or table with the CUDA library and is
@@ -30,7 +30,10 @@
  * of the concatenated batch (brute force); heavy-ball closed form for a
  * constant gradient and the torch.optim.SGD trajectory; finite differences of
  * the loss; controller fixed point, one-step closed form b*tbar/t (Section
- * 3.3), sum conservation, exhaustive check of the integer apportionment.
+ * 3.3), sum conservation, exhaustive check of the integer apportionment;
+ * for the stabilised controller pandas' EWMA, the dead-band at 0.05 and three
+ * traces worked by hand (learnt bounds that cannot hold the global batch, a
+ * bound learnt twice, the smoothed comparison at every observation).
  * Nothing here is left "parity unpinned".
  *
  * Build: gcc -O2 -ffp-contract=off -fopenmp -shared -fPIC (see build.py).

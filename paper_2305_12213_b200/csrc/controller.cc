@@ -164,8 +164,9 @@ extern "C" db_status db_controller_create(db_controller** out, const int32_t* b0
     if (!(kp > 0.0) || !(kp <= 1.0) || !(alpha > 0.0) || !(alpha <= 1.0) || !(dead_band >= 0.0)) return DB_ERR_ARG;
     for (int k = 0; k < K; ++k) {
         if (b0[k] < 1) return DB_ERR_ARG;
-        if (b_min && b_min[k] < 0) return DB_ERR_ARG;
-        if (b_min && b_max && b_max[k] < b_min[k]) return DB_ERR_ARG;
+        // A worker at b = 0 has no iteration time to observe, so the handle's lower bounds start at 1.
+        if (b_min && b_min[k] < 1) return DB_ERR_ARG;
+        if (b_max && b_max[k] < (b_min ? b_min[k] : 1)) return DB_ERR_ARG;
     }
     db_controller* c = new (std::nothrow) db_controller();
     if (!c) return DB_ERR_ARG;

@@ -237,7 +237,44 @@ def test_stabilised_controller_argument_errors(lib):
         E.Controller([4, 4], alpha=0.0)
     with pytest.raises(E.DynbatchError):
         E.Controller([4, 4], dead_band=-1.0)
+    with pytest.raises(E.DynbatchError):
+        E.Controller([4, 4], b_min=[0, 1])          # a worker at b = 0 could never be observed again
+    with pytest.raises(E.DynbatchError):
+        E.Controller([4, 4], b_max=[0, 8])
     c = E.Controller([4, 4])
     with pytest.raises(E.DynbatchError):
         c.observe([1.0, 0.0])
     assert c.observe([1.0, 1.0]) == ([4, 4], False)
+
+
+def test_stabilised_controller_keeps_every_worker_observable_under_strong_heterogeneity(lib):
+    """A 1000:1 throughput ratio would round the slow worker to zero; the lower bound of 1 keeps it
+    alive so that every later observation is still accepted."""
+    c = binding.Controller([8, 8], kp=1.0, alpha=1.0, dead_band=0.0, b_min=[1, 1])
+    b = [8, 8]
+    for _ in range(6):
+        b, _ = c.observe([b[0] / 1000.0, b[1] / 1.0])
+        assert sum(b) == 16 and min(b) >= 1
+    assert b == [15, 1]
+    c.close()
+
+
+HAND_TRACES = [
+    # (b0, kwargs, iteration times per observation, batch sizes expected after each): worked by hand in
+    # tests/test_oracle_pins.py (learnt bounds infeasible; a bound learnt twice; smoothed comparison)
+    ([40, 60], dict(kp=1.0, alpha=1.0, dead_band=0.0, b_max=[65, 100], adaptive_b_max=True),
+     [[8.0, 16.0], [19.0, 10.75], [8.0, 24.0]], [[57, 43], [40, 60], [65, 35]]),
+    ([40, 60], dict(kp=1.0, alpha=1.0, dead_band=0.0, adaptive_b_max=True),
+     [[8.0, 16.0], [19.0, 10.75], [20.0, 10.0], [6.25, 12.5], [16.0, 12.0]],
+     [[57, 43], [40, 60], [25, 75], [40, 60], [25, 75]]),
+    ([40, 60], dict(kp=1.0, alpha=0.5, dead_band=0.35, adaptive_b_max=True),
+     [[8.0, 16.0], [9.0, 10.75], [13.0, 10.75], [14.0, 10.75]],
+     [[57, 43], [57, 43], [57, 43], [40, 60]]),
+]
+
+
+@pytest.mark.parametrize("b0,kw,times,expect", HAND_TRACES)
+def test_stabilised_controller_on_hand_worked_traces(lib, b0, kw, times, expect):
+    c = binding.Controller(b0, **kw)
+    assert [c.observe(t)[0] for t in times] == expect
+    c.close()

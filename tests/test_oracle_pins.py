@@ -471,3 +471,70 @@ def test_adaptive_upper_bound_learns_from_a_throughput_drop():
         plain.observe(times(plain.b))
         seen.append(int(plain.b[0]))
     assert max(seen[2:]) > 100                   # without the learnt bound it keeps crossing the cliff
+
+
+def _trace(st, rows):
+    """Feed iteration times row by row; return (b, learnt_max) after each observation."""
+    out = []
+    for t in rows:
+        st.observe(t)
+        out.append((st.b.tolist(), st.learnt_max.tolist()))
+    return out
+
+
+def test_infeasible_learnt_bounds_fall_back_to_the_users_bounds():
+    """Section 3.3.1, "Batch size bounds", worked by hand (kp = 1, alpha = 1, no dead-band, so every
+    observation readjusts and b' = round(100 * X_k / sum X) within the bounds in force; X_k = b_k / t_k).
+
+    obs 1  b = (40, 60), t = (8, 16)      X = (5, 3.75)  q = (57.14, 42.86)            -> (57, 43)
+    obs 2  b = (57, 43), t = (19, 10.75)  X = (3, 4): worker 0 was raised 40 -> 57 and fell from 5 to 3,
+           so its bound becomes 40.      q = (42.86, 57.14), capped at (40, 100)       -> (40, 60)
+    obs 3  b = (40, 60), t = (8, 24)      X = (5, 2.5): worker 1 was raised 43 -> 60 and fell from 4 to
+           2.5, so its bound becomes 43.  40 + 43 < 100: the learnt bounds cannot hold the global batch,
+           the user's bounds (65, 100) alone apply.  q = (66.67, 33.33), capped at 65  -> (65, 35)
+    """
+    st = oracle.ControllerState([40, 60], kp=1.0, alpha=1.0, dmin=0.0, b_max=[65, 100], adaptive=True)
+    got = _trace(st, [[8.0, 16.0], [19.0, 10.75], [8.0, 24.0]])
+    assert got == [([57, 43], [0, 0]), ([40, 60], [40, 0]), ([65, 35], [40, 43])]
+
+
+def test_a_second_drop_lowers_a_learnt_bound():
+    """Same rules, five observations by hand: the bound learnt at 40 drops to 25 when a later raise
+    from 25 also lowers the throughput, and a raise that does not lower it teaches nothing.
+
+    obs 1  (40, 60), t = (8, 16)       X = (5, 3.75)                                   -> (57, 43)
+    obs 2  (57, 43), t = (19, 10.75)   X = (3, 4)     bound_0 = 40; q_0 = 42.86 capped  -> (40, 60)
+    obs 3  (40, 60), t = (20, 10)      X = (2, 6)     worker 1 raised, but 6 > 4: nothing learnt
+                                                      q = (25, 75)                      -> (25, 75)
+    obs 4  (25, 75), t = (6.25, 12.5)  X = (4, 6)     q = (40, 60)                      -> (40, 60)
+    obs 5  (40, 60), t = (16, 12)      X = (2.5, 5)   worker 0 raised 25 -> 40, fell from 4 to 2.5:
+                                                      bound_0 = 25; q_0 = 33.33 capped  -> (25, 75)
+    """
+    st = oracle.ControllerState([40, 60], kp=1.0, alpha=1.0, dmin=0.0, adaptive=True)
+    got = _trace(st, [[8.0, 16.0], [19.0, 10.75], [20.0, 10.0], [6.25, 12.5], [16.0, 12.0]])
+    assert got == [([57, 43], [0, 0]), ([40, 60], [40, 0]), ([25, 75], [40, 0]),
+                   ([40, 60], [40, 0]), ([25, 75], [25, 0])]
+
+
+def test_learnt_bound_compares_smoothed_throughput_at_every_observation():
+    """alpha = 0.5, dead-band 0.35, by hand.  The comparison uses the smoothed time (a raw-time reading
+    would learn one observation early) and is made at observations that do not readjust as well.
+
+    obs 1  (40, 60), t = (8, 16): first sample, mu = t, X = (5, 3.75), b' = (57, 43); worker 1 moves
+           by 17/60 but worker 0 by 17/40 > 0.35                                        -> readjust
+    obs 2  t = (9, 10.75): first sample since, mu = (9, 10.75), X = (6.33, 4), b' = (61, 39),
+           largest move 4/43                                                            -> keep
+    obs 3  t = (13, 10.75): mu_0 = (13 + 9)/2 = 11, X_0 = 57/11 = 5.18 >= 5: nothing learnt
+           (the raw 57/13 = 4.38 would have); b' = (56, 44)                             -> keep
+    obs 4  t = (14, 10.75): mu_0 = (14 + 11)/2 = 12.5, X_0 = 4.56 < 5 after the raise 40 -> 57:
+           bound_0 = 40; q_0 = 53.27 capped at 40, b' = (40, 60), moves 17/57 and 17/43 -> readjust
+           (without the bound b' = (53, 47), inside the dead-band)
+    """
+    st = oracle.ControllerState([40, 60], kp=1.0, alpha=0.5, dmin=0.35, adaptive=True)
+    assert st.observe([8.0, 16.0]) is True and st.b.tolist() == [57, 43]
+    assert st.observe([9.0, 10.75]) is False and st.ewma.tolist() == [9.0, 10.75]
+    assert st.observe([13.0, 10.75]) is False
+    assert st.ewma.tolist() == [11.0, 10.75] and st.learnt_max.tolist() == [0, 0]
+    assert st.b.tolist() == [57, 43]
+    assert st.observe([14.0, 10.75]) is True
+    assert st.learnt_max.tolist() == [40, 0] and st.b.tolist() == [40, 60]
