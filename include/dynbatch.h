@@ -14,9 +14,12 @@
  *     synchronising.  Host arrays (batch sizes, pointer tables) are consumed
  *     before the call returns.
  *   - Every call returns a db_status.  Arguments are validated before any
- *     launch; on an error nothing has been enqueued and no output is touched.
+ *     launch; on an argument error (DB_ERR_NULL / ARG / UNSUPPORTED /
+ *     INFEASIBLE) nothing has been enqueued and no output is touched.
  *     Nothing throws, aborts or traps.  After DB_ERR_CUDA,
- *     db_last_cuda_error() returns the runtime's message for this thread.
+ *     db_last_cuda_error() returns the runtime's message for this thread; an
+ *     entry point that enqueues several operations may then have enqueued
+ *     some of them, and outputs are unspecified.
  *   - NaN/Inf in the inputs propagate by IEEE rules; they are not checked.
  */
 #ifndef DYNBATCH_H_

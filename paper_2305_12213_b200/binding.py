@@ -18,6 +18,7 @@ import torch
 DB_OK, DB_ERR_NULL, DB_ERR_ARG, DB_ERR_UNSUPPORTED, DB_ERR_INFEASIBLE, DB_ERR_CUDA = range(6)
 DB_F32, DB_BF16 = 0, 1
 DB_MAX_K = 64
+DB_STATIC_SCRATCH_BYTES = 1 << 20     # the built-in scratch of aggregate_update_static
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libdynbatch.so")
 

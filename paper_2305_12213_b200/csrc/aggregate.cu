@@ -502,8 +502,18 @@ extern "C" db_status db_aggregate_update_static(const void* const* grads, db_dty
                                                 float* momentum, float lr, float mu,
                                                 double* grad_sqnorm, void* cuda_stream) {
     using namespace dynbatch;
+    // the cheap argument checks first, so that a bad call is reported as what it is, not as too large
+    if (!grads || !b || !params || !momentum) return DB_ERR_NULL;
+    if (K < 1 || K > DB_MAX_K || N < 0) return DB_ERR_ARG;
+    if (grad_dtype != DB_F32 && grad_dtype != DB_BF16) return DB_ERR_UNSUPPORTED;
+    long long total = 0;
+    for (int k = 0; k < K; ++k) {
+        if (b[k] < 0) return DB_ERR_ARG;
+        total += b[k];
+    }
+    if (total <= 0 || !isfinite(lr) || !isfinite(mu)) return DB_ERR_ARG;
     void* scratch = nullptr;
-    if (grad_sqnorm) {
+    if (grad_sqnorm && N > 0) {
         const size_t need = db_aggregate_workspace_bytes(K, N);
         if (need > DB_STATIC_SCRATCH_BYTES) {
             char msg[256];

@@ -8,6 +8,7 @@
 // stream), so that PCIe runs in both directions while the kernel works on the
 // previous chunk.  Two staging slots in device memory hold the chunks in flight.
 #include <cstdint>
+#include <cmath>
 #include <new>
 
 #include "common.h"
@@ -127,52 +128,76 @@ extern "C" db_status db_aggregate_update_host(db_host_pipeline* h, const void* c
     double* total_norm = reinterpret_cast<double*>(base + L.total_off);
     const int64_t nchunks = (N + chunk - 1) / chunk;
 
+    // Everything that can be rejected is rejected here, before the first event is recorded: an error
+    // from an argument leaves nothing enqueued on any stream.
+    if (!std::isfinite(lr) || !std::isfinite(mu)) return DB_ERR_ARG;
+    if (reinterpret_cast<uintptr_t>(params) % 4 || reinterpret_cast<uintptr_t>(momentum) % 4) return DB_ERR_ARG;
+    {
+        const uintptr_t p0 = reinterpret_cast<uintptr_t>(params), v0 = reinterpret_cast<uintptr_t>(momentum);
+        const uintptr_t s0 = reinterpret_cast<uintptr_t>(staging);
+        const size_t state_bytes = static_cast<size_t>(N) * 4;
+        auto overlap = [](uintptr_t a, size_t an, uintptr_t c, size_t cn) { return a < c + cn && c < a + an; };
+        if (overlap(p0, state_bytes, v0, state_bytes) || overlap(p0, state_bytes, s0, L.end) ||
+            overlap(v0, state_bytes, s0, L.end))
+            return DB_ERR_ARG;
+    }
+
     // Everything below is ordered after the caller's earlier work on its stream.
     DB_CUDA_TRY(cudaEventRecord(h->start, compute));
     DB_CUDA_TRY(cudaStreamWaitEvent(h->in, h->start, 0));
     DB_CUDA_TRY(cudaStreamWaitEvent(h->out, h->start, 0));
 
-    for (int64_t c = 0; c < nchunks; ++c) {
-        const int s = static_cast<int>(c % kSlots);
-        const int64_t off = c * chunk;
-        const int64_t len = (N - off < chunk) ? (N - off) : chunk;
-        char* slot = base + L.slots_off + s * L.slot_bytes;
-        const void* slices[DB_MAX_K];
+    auto enqueue_chunks = [&]() -> db_status {
+        for (int64_t c = 0; c < nchunks; ++c) {
+            const int s = static_cast<int>(c % kSlots);
+            const int64_t off = c * chunk;
+            const int64_t len = (N - off < chunk) ? (N - off) : chunk;
+            char* slot = base + L.slots_off + s * L.slot_bytes;
+            const void* slices[DB_MAX_K];
 
-        // copy-in: the slot is free once the kernel that read it two chunks ago has finished
-        if (c >= kSlots) DB_CUDA_TRY(cudaStreamWaitEvent(h->in, h->computed[s], 0));
-        for (int k = 0; k < K; ++k) {
-            char* dst = slot + static_cast<size_t>(k) * chunk * gsize;
-            slices[k] = dst;
-            if (b[k] == 0) continue;  // weight 0: neither copied nor read
-            DB_CUDA_TRY(cudaMemcpyAsync(dst, static_cast<const char*>(host_grads[k]) + off * gsize,
-                                        static_cast<size_t>(len) * gsize, cudaMemcpyHostToDevice, h->in));
+            // copy-in: the slot is free once the kernel that read it two chunks ago has finished
+            if (c >= kSlots) DB_CUDA_TRY(cudaStreamWaitEvent(h->in, h->computed[s], 0));
+            for (int k = 0; k < K; ++k) {
+                char* dst = slot + static_cast<size_t>(k) * chunk * gsize;
+                slices[k] = dst;
+                if (b[k] == 0) continue;  // weight 0: neither copied nor read
+                DB_CUDA_TRY(cudaMemcpyAsync(dst, static_cast<const char*>(host_grads[k]) + off * gsize,
+                                            static_cast<size_t>(len) * gsize, cudaMemcpyHostToDevice, h->in));
+            }
+            DB_CUDA_TRY(cudaEventRecord(h->loaded[s], h->in));
+
+            // compute on the caller's stream
+            DB_CUDA_TRY(cudaStreamWaitEvent(compute, h->loaded[s], 0));
+            long long ctas = 0;
+            const db_status st = aggregate_chunk(slices, grad_dtype, b, K, len, params + off, momentum + off, lr, mu,
+                                                 host_sqnorm_out ? partials + n_partials : nullptr, &ctas, compute);
+            if (st != DB_OK) return st;
+            n_partials += ctas;
+            DB_CUDA_TRY(cudaEventRecord(h->computed[s], compute));
+
+            // copy-out of the updated parameters
+            if (host_params_out) {
+                DB_CUDA_TRY(cudaStreamWaitEvent(h->out, h->computed[s], 0));
+                DB_CUDA_TRY(cudaMemcpyAsync(host_params_out + off, params + off, static_cast<size_t>(len) * 4,
+                                            cudaMemcpyDeviceToHost, h->out));
+            }
         }
-        DB_CUDA_TRY(cudaEventRecord(h->loaded[s], h->in));
-
-        // compute on the caller's stream
-        DB_CUDA_TRY(cudaStreamWaitEvent(compute, h->loaded[s], 0));
-        long long ctas = 0;
-        const db_status st = aggregate_chunk(slices, grad_dtype, b, K, len, params + off, momentum + off, lr, mu,
-                                             host_sqnorm_out ? partials + n_partials : nullptr, &ctas, compute);
-        if (st != DB_OK) return st;
-        n_partials += ctas;
-        DB_CUDA_TRY(cudaEventRecord(h->computed[s], compute));
-
-        // copy-out of the updated parameters
-        if (host_params_out) {
-            DB_CUDA_TRY(cudaStreamWaitEvent(h->out, h->computed[s], 0));
-            DB_CUDA_TRY(cudaMemcpyAsync(host_params_out + off, params + off, static_cast<size_t>(len) * 4,
-                                        cudaMemcpyDeviceToHost, h->out));
+        if (host_sqnorm_out) {
+            const db_status st = finalize_norm(partials, n_partials, total_norm, compute);
+            if (st != DB_OK) return st;
+            DB_CUDA_TRY(cudaMemcpyAsync(host_sqnorm_out, total_norm, sizeof(double), cudaMemcpyDeviceToHost, compute));
         }
-    }
-    if (host_sqnorm_out) {
-        const db_status st = finalize_norm(partials, n_partials, total_norm, compute);
-        if (st != DB_OK) return st;
-        DB_CUDA_TRY(cudaMemcpyAsync(host_sqnorm_out, total_norm, sizeof(double), cudaMemcpyDeviceToHost, compute));
-    }
-    // the caller's stream completes only after the last parameter chunk has reached the host
-    DB_CUDA_TRY(cudaEventRecord(h->drained, h->out));
-    DB_CUDA_TRY(cudaStreamWaitEvent(compute, h->drained, 0));
+        return DB_OK;
+    };
+    const db_status st = enqueue_chunks();
+    // The caller's stream completes only after everything queued on the two copy streams has: the last
+    // parameter chunk has reached the host, and -- should a CUDA call have failed half way -- no copy of this
+    // call is still in flight when the caller's stream moves on.
+    cudaError_t join = cudaEventRecord(h->loaded[0], h->in);
+    if (join == cudaSuccess) join = cudaStreamWaitEvent(compute, h->loaded[0], 0);
+    if (join == cudaSuccess) join = cudaEventRecord(h->drained, h->out);
+    if (join == cudaSuccess) join = cudaStreamWaitEvent(compute, h->drained, 0);
+    if (st != DB_OK) return st;
+    DB_CUDA_TRY(join);
     return DB_OK;
 }

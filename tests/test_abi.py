@@ -42,6 +42,12 @@ def test_binding_covers_every_symbol(lib):
     assert sorted(binding._SIGNATURES) == _declared_symbols()
 
 
+def test_binding_constants_are_the_headers(lib):
+    text = open(os.path.join(ROOT, "include", "dynbatch.h")).read()
+    for name in ("DB_MAX_K", "DB_STATIC_SCRATCH_BYTES"):
+        assert int(re.search(rf"#define\s+{name}\s+(\d+)", text).group(1)) == getattr(binding, name)
+
+
 def test_status_strings(lib):
     assert lib.db_status_string(0) == b"ok"
     assert len({lib.db_status_string(i) for i in range(6)}) == 6

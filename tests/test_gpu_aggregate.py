@@ -324,7 +324,7 @@ def test_config_bert_base_sixteen_workers_bf16():
         return X
 
     b, worst = _iterate(16, N, torch.bfloat16, 1e-3, [32] * 16, X_of, 1.0, 0.05, 0.9, 200, 3000,
-                        full_at={0, 50, 199}, sample=1 << 20)
+                        full_at={0, 1, 2, 49, 50, 51, 52, 199}, sample=1 << 20)
     assert sum(b) == 512
     want = 512 * np.array(X_of(199)) / sum(X_of(199))
     assert np.abs(np.array(b) - want).max() <= 1.0

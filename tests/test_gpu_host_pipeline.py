@@ -62,4 +62,16 @@ def test_optional_outputs_and_errors():
     assert ei.value.status == binding.DB_ERR_ARG
     with pytest.raises(binding.DynbatchError):
         pipe.aggregate_update(pinned, [0, 0], p, v, 1.0, 0.0, None, None, staging, 4096)
+    # params and momentum that overlap, or a non-finite step size: rejected before anything is
+    # enqueued, so the state is untouched and the pipeline is still usable
+    before = v.clone()
+    for args in ((p, p[: N // 2], 1.0), (v, v, 1.0), (p, v, float("nan"))):
+        with pytest.raises(binding.DynbatchError) as ei:
+            pipe.aggregate_update([g[: args[1].numel()] for g in pinned], [1, 1], args[0][: args[1].numel()],
+                                  args[1], args[2], 0.0, None, None, staging, 4096)
+        assert ei.value.status == binding.DB_ERR_ARG
+    torch.cuda.synchronize()
+    assert torch.equal(v, before)
+    pipe.aggregate_update(pinned, [1, 1], p, v, 1.0, 0.0, None, None, staging, 4096)
+    torch.cuda.synchronize()
     pipe.close()

@@ -50,8 +50,9 @@ def test_matches_per_tensor_calls_and_oracle(dtype, shift):
         torch.cuda.synchronize()
         for t in range(len(sizes)):
             assert torch.equal(params[t], ref_p[t]) and torch.equal(momentum[t], ref_v[t]), f"tensor {t} step {step}"
-            assert rel_err(f64(params[t]), p0[t]) <= FP32_TOL * (step + 1)
-            assert rel_err(f64(momentum[t]), v0[t]) <= FP32_TOL * (step + 1)
+            # the oracle keeps its own fp64 state over both steps (free-running), same gate as one step
+            assert rel_err(f64(params[t]), p0[t]) <= FP32_TOL
+            assert rel_err(f64(momentum[t]), v0[t]) <= FP32_TOL
         assert abs(float(sq.item()) - total) <= FP32_TOL * total
     plan.close()
 
@@ -77,17 +78,6 @@ def test_resnet50_tensor_list_equals_the_flat_arena_call():
     torch.cuda.synchronize()
     assert torch.equal(p1, p2) and torch.equal(v1, v2)
     assert abs(float(sq1.item()) - float(sq2.item())) <= 1e-9 * float(sq1.item())
-    # timing, reported only: one launch over 161 tensors against the flat call
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    for fn in (lambda: plan.step(b, 0.1, 0.9, sq2), lambda: binding.aggregate_update(g, b, p1, v1, 0.1, 0.9, sq1, ws)):
-        for _ in range(3):
-            fn()
-        e0.record()
-        for _ in range(20):
-            fn()
-        e1.record()
-        torch.cuda.synchronize()
-        print(f"{e0.elapsed_time(e1) / 20 * 1e3:.1f} us per step")
     plan.close()
 
 
