@@ -115,6 +115,24 @@ def copy_probe(dev, nbytes: int = 1 << 30, reps: int = 10) -> float:
     return 2.0 * nbytes * reps / (e0.elapsed_time(e1) * 1e-3) / 1e9
 
 
+def read_probe(dev, nbytes: int = 1 << 30, reps: int = 10) -> float:
+    """GB/s of a pure read stream over 1 GiB (the library's own probe kernel, 128-bit streaming loads)."""
+    from paper_2305_12213_b200 import binding
+    src = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    src.zero_()
+    sink = torch.empty(binding.bench_read_probe_sink_bytes(nbytes), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    for _ in range(3):
+        binding.bench_read_probe(src, sink, stream)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(reps):
+        binding.bench_read_probe(src, sink, stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return float(nbytes) * reps / (e0.elapsed_time(e1) * 1e-3) / 1e9
+
+
 def step_bytes(K: int, N: int, grad_bytes: int) -> int:
     """Algorithmic HBM bytes of one step: K gradient reads + read and write of params and momentum."""
     return K * N * grad_bytes + 4 * N * 4
@@ -150,7 +168,7 @@ class ClockSampler:
     REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
                0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
 
-    def __init__(self, index: int, period_s: float = 0.005):
+    def __init__(self, index: int, period_s: float = 0.001):
         self.samples, self.reasons = [], set()
         self.max_mhz = None
         self._stop = threading.Event()
@@ -234,6 +252,13 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
         cut = lambda t: [t[s:e] for s, e in zip(offs[:-1], offs[1:])]
         plan = binding.MultiTensorPlan([cut(g) for g in grads], cut(p), cut(v))
         kernel_label = f"agg_multi_kernel over {len(shapes)} tensors"
+    elif variant in ("persistent", "staged"):
+        # the launch shapes that were measured against the kept kernel and not adopted (no norm)
+        if wl.grad_dtype != torch.float32 or K not in (2, 4, 8, 16) or N % 4:
+            raise SystemExit(f"--variant {variant} covers fp32 gradients, K in 2, 4, 8, 16 and N % 4 == 0")
+        vstatus = torch.zeros(1, dtype=torch.int32, device=dev)
+        kernel_label = "persistent_kernel" if variant == "persistent" else f"bulk_staged_kernel[{args.stage_floats} floats]"
+    with_norm = variant in ("momentum", "adam", "tensor_list")
 
     def step():
         nonlocal b, adam_t
@@ -243,6 +268,12 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
             binding.aggregate_adam(grads, b, p, v, u, 1e-3, 0.9, 0.999, 1e-8, adam_t, sq, ws, stream)
         elif variant == "tensor_list":
             plan.step(b, wl.lr, wl.mu, sq, stream)
+        elif variant == "nonorm":
+            binding.aggregate_update(grads, b, p, v, wl.lr, wl.mu, None, None, stream)
+        elif variant in ("persistent", "staged"):
+            binding.bench_aggregate_variant(
+                binding.DB_BENCH_PERSISTENT if variant == "persistent" else binding.DB_BENCH_BULK_STAGED,
+                args.stage_floats, grads, b, p, v, wl.lr, wl.mu, vstatus, stream)
         else:
             binding.aggregate_update(grads, b, p, v, wl.lr, wl.mu, sq, ws, stream)
 
@@ -258,21 +289,21 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
     torch.cuda.synchronize()
     if flush is None:
         e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        with sampler:
+        n_probe = min(steps, 200)
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_probe)]
+        with sampler:             # the clocks are sampled through the timed region and the per-call pass behind it
             e_begin.record(stream)
             for _ in range(steps):
                 step()
             e_end.record(stream)
             torch.cuda.synchronize()
+            # the kernel's own duration: a second pass with an event pair around every call
+            for e0, e1 in pairs:
+                e0.record(stream)
+                step()
+                e1.record(stream)
+            torch.cuda.synchronize()
         elapsed_ms = e_begin.elapsed_time(e_end)
-        # the kernel's own duration: a second pass with an event pair around every call
-        n_probe = min(steps, 200)
-        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_probe)]
-        for e0, e1 in pairs:
-            e0.record(stream)
-            step()
-            e1.record(stream)
-        torch.cuda.synchronize()
         per_step_ms = [e0.elapsed_time(e1) for e0, e1 in pairs]
     else:
         pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
@@ -291,8 +322,12 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
     replicas.barrier(dev)
     bytes_step = wl.K * wl.N * wl.grad_bytes + state_bytes * wl.N
     job_bps, max_ms = replicas.job_throughput(bytes_step * steps, elapsed_ms, dev)
-    final_sq = float(sq.item())
-    assert np.isfinite(final_sq) and final_sq > 0 and bool(torch.isfinite(p[:1024]).all())
+    if with_norm:
+        final_sq = float(sq.item())
+        assert np.isfinite(final_sq) and final_sq > 0
+    if variant in ("persistent", "staged"):
+        assert int(vstatus.item()) == 0, "a staged CTA gave up waiting for its copies"
+    assert bool(torch.isfinite(p[:1024]).all())
 
     peak, peak_kind = measured_peak()
     # The dominant kernel's launch duration, from CUDA events on its stream.  Back-to-back mode: the timed
@@ -302,25 +337,29 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
     kernel_ms = elapsed_ms / steps if flush is None else float(np.mean(per_step_ms))
     achieved = bytes_step / (kernel_ms * 1e-3) / 1e9
     gname = "float" if wl.grad_dtype == torch.float32 else "__nv_bfloat16"
+    launches = 2 if with_norm else 1
     out = {
         "metric": METRIC if variant == "momentum" else f"{METRIC} [{variant} variant of the step]",
         "value": job_bps / 1e9, "unit": "GB/s",
         "iterations_per_s": world * steps / (max_ms * 1e-3),
         "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": max_ms / steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "vs_baseline": None,
+        "dtype": "f32" if wl.grad_dtype == torch.float32 else "bf16 gradients, f32 accumulation and state",
+        "data": "synthetic",
         "config": {"workload": wl.name if variant == "momentum" else f"{wl.name}_{variant}", "K": K, "N": N,
                    "grad_dtype": "f32" if wl.grad_dtype == torch.float32 else "bf16",
-                   "global_batch": sum(wl.b0), "kp": wl.kp, "lr": wl.lr, "mu": wl.mu, "grad_sqnorm": True,
+                   "global_batch": sum(wl.b0), "kp": wl.kp, "lr": wl.lr, "mu": wl.mu, "grad_sqnorm": with_norm,
                    "bytes_per_step": bytes_step,
                    "l2": ("inputs (%.2f GB per step) exceed the 126 MB L2" % (wl.working_set / 1e9)) if flush is None
                    else "L2 flushed (252 MB written, then read) before every timed step",
                    "parallelism": f"{world} independent replica(s), no collective"},
-        "gpu_launches": 2 * steps,  # the aggregation kernel and the one-CTA fold of its norm partials
+        # the aggregation kernel, plus the one-CTA fold of its norm partials scheduled under it
+        "gpu_launches": launches * steps,
         "clocks": sampler.summary(),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": f"of {peak_kind}",
-                     "kernel": f"{kernel_label}<{gname}, K={K if K <= 16 else 0}, norm, {'adam' if variant == 'adam' else 'momentum'}>",
+                     "kernel": f"{kernel_label}<{gname}, K={K if K <= 16 else 0}, {'norm' if with_norm else 'no norm'}, {'adam' if variant == 'adam' else 'momentum'}>",
                      "kernel_ms": kernel_ms,
                      "kernel_ms_probe_mean": float(np.mean(per_step_ms)),
                      "kernel_ms_min": float(np.min(per_step_ms)),
@@ -333,6 +372,7 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
     if with_e2e:
         # context only: this run's own device-to-device copy, the kind of measurement the peak file holds
         out["roofline"]["copy_probe_gbs"] = copy_probe(dev)
+        out["roofline"]["read_probe_gbs"] = read_probe(dev)
         out["e2e"] = measure_e2e(wl, args, dev, grads, p, v, b)
     if with_cpu and rank == 0 and world == 1:
         out["cpu_baseline"] = cpu_baseline(wl, host_gradients(grads), b)
@@ -442,7 +482,9 @@ def measure_softmax(args, dev, rank, world):
         "config": {"workload": "softmax_D2048_C1000_b24_40_64_128", "D": D, "C": C, "batch_sizes": bs,
                    "l2": "L2 flushed (252 MB written, then read) before every timed step",
                    "calls": "db_worker_grad_grouped + db_aggregate_update_ex"},
-        "gpu_launches": 5 * steps, "clocks": sampler.summary(),   # logits, softmax, gradients, aggregation, norm fold
+        # logits, softmax, gradients, aggregation, norm fold
+        "gpu_launches": 5 * steps,
+        "clocks": sampler.summary(),
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak, "peak_source": kind,
                      "note": "algorithmic FLOPs 4*sum(b)*D*C per step; the step is launch- and latency-bound "
@@ -496,23 +538,38 @@ def host_gradients(grads):
     return out
 
 
-def cpu_baseline(wl, host_grads, b, budget_s: float = 15.0):
-    """The fp64 oracle, as it stands, on the host cores, over the same workload (all N, all K)."""
+def cpu_baseline(wl, host_grads, b, budget_s: float = 12.0):
+    """The fp64 oracle, as it stands, on the host cores, over the same workload (all N, all K): with all
+    cores, and with one thread."""
     import oracle
     N = wl.N
     p = inputs.normal(N, PARAM_STD, 1, "cpu").numpy().astype(np.float64)
     v = np.zeros(N, dtype=np.float64)
-    oracle.aggregate_update(host_grads, b, p, v, wl.lr, wl.mu)          # warm-up pass
-    t0 = time.perf_counter()
-    passes = 0
-    while passes < 3 or (time.perf_counter() - t0 < budget_s and passes < 50):
-        oracle.aggregate_update(host_grads, b, p, v, wl.lr, wl.mu)
-        passes += 1
-    dt = time.perf_counter() - t0
-    return {"value": wl.bytes_per_step * passes / dt / 1e9, "unit": "GB/s", "cores": oracle.num_threads(),
-            "kind": "oracle", "iterations_per_s": passes / dt,
+    all_threads = oracle.num_threads()
+
+    def timed(threads, budget, min_passes):
+        oracle.set_num_threads(threads)
+        oracle.aggregate_update(host_grads, b, p, v, wl.lr, wl.mu)          # warm-up pass
+        t0 = time.perf_counter()
+        passes = 0
+        while passes < min_passes or (time.perf_counter() - t0 < budget and passes < 50):
+            oracle.aggregate_update(host_grads, b, p, v, wl.lr, wl.mu)
+            passes += 1
+        dt = time.perf_counter() - t0
+        return passes, dt
+
+    try:
+        passes, dt = timed(all_threads, budget_s, 3)
+        passes1, dt1 = timed(1, budget_s / 2, 1)
+    finally:
+        oracle.set_num_threads(all_threads)
+    return {"value": wl.bytes_per_step * passes / dt / 1e9, "unit": "GB/s", "cores": all_threads,
+            "kind": "oracle", "iterations_per_s": passes / dt, "ms_per_iteration": dt / passes * 1e3,
             "sample": f"{passes} full passes of the workload (N={N}, K={wl.K}), "
-                      "fp64 state, OpenMP over elements"}
+                      "fp64 state, OpenMP over elements",
+            "single_thread": {"value": wl.bytes_per_step * passes1 / dt1 / 1e9, "unit": "GB/s", "cores": 1,
+                              "ms_per_iteration": dt1 / passes1 * 1e3,
+                              "sample": f"{passes1} full pass(es) of the same workload"}}
 
 
 def run_reference(args):
@@ -550,6 +607,15 @@ def run_reference(args):
     dt = time.perf_counter() - t0
     val = step_bytes(K, n, wl.grad_bytes) * steps / dt / 1e9
     sample = f"first {n} of {N} parameters per step, all K={K} workers, fp64 state"
+    # the same sample once on a single thread, outside the timed region
+    all_threads = oracle.num_threads()
+    oracle.set_num_threads(1)
+    try:
+        t1 = time.perf_counter()
+        step()
+        dt1 = time.perf_counter() - t1
+    finally:
+        oracle.set_num_threads(all_threads)
     out = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s",
         "iterations_per_s": (n / N) * steps / dt,
@@ -559,8 +625,10 @@ def run_reference(args):
         "config": {"workload": wl.name, "K": K, "N": N,
                    "grad_dtype": "f32" if wl.grad_dtype == torch.float32 else "bf16",
                    "global_batch": sum(wl.b0), "kp": wl.kp, "lr": wl.lr, "mu": wl.mu, "sample": sample},
-        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle",
-                         "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": all_threads, "kind": "oracle",
+                         "sample": sample,
+                         "single_thread": {"value": step_bytes(K, n, wl.grad_bytes) / dt1 / 1e9, "unit": "GB/s",
+                                           "cores": 1, "sample": "one step of the same sample"}},
         "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -573,10 +641,15 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--variant", choices=["momentum", "adam", "tensor_list"], default="momentum",
-                    help="the step's optimizer / entry point (resnet50 and bert_base workloads): momentum = "
-                         "db_aggregate_update_ex (headline), adam = db_aggregate_adam_ex, tensor_list = "
-                         "db_aggregate_update_multi over the model's separate tensors")
+    ap.add_argument("--variant", choices=["momentum", "adam", "tensor_list", "nonorm", "persistent", "staged"],
+                    default="momentum",
+                    help="the step's optimizer / entry point: momentum = db_aggregate_update_ex (headline), adam = "
+                         "db_aggregate_adam_ex, tensor_list = db_aggregate_update_multi over the model's separate "
+                         "tensors (resnet50, bert_base); nonorm = the headline kernel without the gradient norm, "
+                         "persistent / staged = the launch shapes measured against it and not adopted "
+                         "(db_bench_aggregate_variant; fp32, no norm)")
+    ap.add_argument("--stage-floats", type=int, choices=[512, 1024, 2048], default=512,
+                    help="with --variant staged: floats per stream and CTA staged in shared memory")
     ap.add_argument("--sweep-dtype", choices=["fp32", "bf16"], default="fp32",
                     help="gradient storage of the sweep's points (the named sweep configuration is fp32)")
     ap.add_argument("--sweep-point", default="", metavar="N,K",

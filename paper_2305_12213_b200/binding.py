@@ -50,6 +50,10 @@ _SIGNATURES = {
     "db_multi_plan_destroy": (c_int32, [c_void_p]),
     "db_aggregate_update_static": (c_int32, [c_void_p, c_int32, c_void_p, c_int32, c_int64, c_void_p,
                                              c_void_p, c_float, c_float, c_void_p, c_void_p]),
+    "db_bench_read_probe_sink_bytes": (c_size_t, [c_size_t]),
+    "db_bench_read_probe": (c_int32, [c_void_p, c_size_t, c_void_p, c_void_p]),
+    "db_bench_aggregate_variant": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_int32, c_int64, c_void_p,
+                                             c_void_p, c_float, c_float, c_void_p, c_void_p]),
     "db_host_pipeline_create": (c_int32, [c_void_p]),
     "db_host_pipeline_destroy": (c_int32, [c_void_p]),
     "db_host_staging_bytes": (c_size_t, [c_int32, c_int32, c_int64, c_int64]),
@@ -200,6 +204,38 @@ def aggregate_update_static(grads: Sequence[torch.Tensor], b: Sequence[int], par
         ctypes.cast(_i32_array(b), c_void_p), K, int(params.numel()),
         _dev_ptr(params, torch.float32, "params"), _dev_ptr(momentum, torch.float32, "momentum"),
         float(lr), float(mu), _dev_ptr(grad_sqnorm, torch.float64, "grad_sqnorm"), _stream_ptr(stream)))
+
+
+DB_BENCH_PERSISTENT, DB_BENCH_BULK_STAGED = 1, 2
+
+
+def bench_read_probe_sink_bytes(nbytes: int) -> int:
+    return int(lib().db_bench_read_probe_sink_bytes(int(nbytes)))
+
+
+def bench_read_probe(src: torch.Tensor, sink: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """db_bench_read_probe: stream all of `src` through registers once (a measurement helper)."""
+    if not (src.is_cuda and sink.is_cuda and src.is_contiguous() and sink.is_contiguous()):
+        raise TypeError("src and sink must be contiguous CUDA tensors")
+    nbytes = src.numel() * src.element_size()
+    if sink.numel() * sink.element_size() < bench_read_probe_sink_bytes(nbytes):
+        raise ValueError("sink too small")
+    _check(lib().db_bench_read_probe(src.data_ptr(), nbytes, sink.data_ptr(), _stream_ptr(stream)))
+
+
+def bench_aggregate_variant(variant: int, stage_floats: int, grads: Sequence[torch.Tensor], b: Sequence[int],
+                            params: torch.Tensor, momentum: torch.Tensor, lr: float, mu: float,
+                            status: Optional[torch.Tensor] = None,
+                            stream: Optional[torch.cuda.Stream] = None) -> None:
+    """db_bench_aggregate_variant: the momentum step in a launch shape that was measured and not adopted."""
+    K = len(grads)
+    if len(b) != K:
+        raise ValueError("len(b) != len(grads)")
+    table = (c_void_p * K)(*[_dev_ptr(g, torch.float32, "grads[k]") for g in grads])
+    _check(lib().db_bench_aggregate_variant(
+        int(variant), int(stage_floats), ctypes.cast(table, c_void_p), ctypes.cast(_i32_array(b), c_void_p), K,
+        int(params.numel()), _dev_ptr(params, torch.float32, "params"), _dev_ptr(momentum, torch.float32, "momentum"),
+        float(lr), float(mu), _dev_ptr(status, torch.int32, "status"), _stream_ptr(stream)))
 
 
 def _dtype_code(dt: torch.dtype) -> int:

@@ -48,6 +48,7 @@ struct GemmArgs {
     int k_per_split;                        // multiple of kBlockK; split z covers [z*kps, min(K, (z+1)*kps))
     int n_acc;                              // main accumulators used round-robin, (n_acc + 1) * N_TILE <= 512
     int* status;                            // device word, set non-zero if a wait gave up
+    int clear_status;                       // non-zero: the first CTA zeroes *status before any wait can set it
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -355,6 +356,8 @@ __device__ __forceinline__ void tf32x3_gemm_body(const GemmArgs& g, const int sp
     // everything above overlaps the previous kernel; its outputs are read only from here on
     griddep_launch_dependents();
     griddep_wait();
+    // a time-out needs seconds, this store comes microseconds after the launch: no wait can have given up yet
+    if (g.clear_status && tid == 0 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) *g.status = 0;
 
     if (warp < kLoaderWarps) {
         // ------------------------------------------------------------ producers

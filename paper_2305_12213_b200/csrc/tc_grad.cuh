@@ -6,23 +6,31 @@
 // tc_gemm.cuh has to do; what is left of the operand preparation, the split of every fp32 value
 // into two TF32 halves, is done once by the kernel that produces E (and copies X), not once per
 // output tile.  A CTA of this kernel therefore only
-//   - copies [16 rows x 32 columns] boxes of the four split arrays (X_hi, X_lo, E_hi, E_lo) into
-//     shared memory with cp.async.bulk.tensor (128-byte swizzle of 32-byte pieces, completion on an
-//     mbarrier),
+//   - copies boxes of 16 rows of the four split arrays (X_hi, X_lo, E_hi, E_lo) into shared memory
+//     with cp.async.bulk.tensor (128-byte swizzle of 32-byte pieces, completion on an mbarrier),
 //   - issues three tcgen05.mma.kind::tf32 per 8 rows (lo*hi + hi*lo into one accumulator in tensor
-//     memory, hi*hi round-robin into up to seven others, see tc_gemm.cuh for why), and
-//   - drains the accumulators and writes its 128 x 64 tile of G: through shared memory in the box
-//     layout of a TMA store when G is 16-byte aligned with rows of a multiple of 16 bytes, else as
-//     whole rows with ordinary stores.
+//     memory, hi*hi round-robin into the others, see tc_gemm.cuh for why), and
+//   - drains the accumulators and writes its 128 x TILE_N tile of G: through shared memory in the
+//     box layout of a TMA store when G is 16-byte aligned with rows of a multiple of 16 bytes, else
+//     as whole rows with ordinary stores.
 // In the split arrays every worker's rows start at a multiple of 8 and are padded with zero rows to
 // a multiple of 8, the reduction depth of one TF32 product.
 //
+// What bounds the kernel is the stream of operand tiles from the L2 (measured: about 10 TB/s while
+// the copy loops run, for operands that total a few MB but are re-read by every tile), so
+//   - the tile is 128 x 128 where the accumulator chains allow it (batches up to 1024 rows; two
+//     thirds of the operand traffic of 128 x 64 tiles), else 128 x 64 with up to seven accumulators;
+//   - the workers are dealt into groups (largest first, each to the lightest group) and a CTA works
+//     through all workers of its group for one tile, so that the whole grid is resident at once where
+//     the sizes allow it: with one CTA per worker and tile the small workers' CTAs formed a second
+//     wave that started only when the large workers' CTAs retired.
+//
 // 192 threads: warp 0 (one lane) issues the TMA copies, warp 1 owns the tensor-memory allocation
-// and (one lane) issues the products, warps 2-5 are the epilogue.  Two shared-memory stages of
-// 24 KB (16 samples each), so four CTAs fit on an SM and their phases (copy, products, epilogue)
-// overlap; measured, a CTA's own phases are latency-bound and more resident CTAs pay.  Every wait is
-// bounded (see tc_gemm.cuh); on a time-out the copy thread waits, again bounded, for the copies it
-// has in flight before the CTA returns.
+// and (one lane) issues the products, warps 2-5 are the epilogue.  Three shared-memory stages of
+// 16 samples.  Between two workers of a group the copy thread and the issuing thread wait until the
+// epilogue has drained the accumulators and stored the tile (the staging tile reuses the operand
+// stages).  Every wait is bounded (see tc_gemm.cuh); on a time-out the copy thread waits, again
+// bounded, for the copies it has in flight before the CTA returns.
 #pragma once
 #include <cuda.h>
 
@@ -32,37 +40,54 @@ namespace dynbatch {
 namespace tcg {
 
 constexpr int kTileM = 128;            // features per CTA = tensor-memory lanes
-constexpr int kTileN = 64;             // classes per CTA = accumulator columns
 constexpr int kChunk = 32;             // fp32 per 128-byte swizzled row
 constexpr int kStepRows = 8;           // reduction depth of one TF32 product
 constexpr int kRowsPerStage = 16;      // samples per stage: two products' worth
 constexpr int kAccRows = 32;           // consecutive samples whose hi*hi products share an accumulator turn
-constexpr int kStages = 2;
-constexpr int kChunkBytes = kRowsPerStage * 128;            // one [16 x 32] box
-constexpr int kAChunks = kTileM / kChunk, kBChunks = kTileN / kChunk;
+constexpr int kStages = 3;
+constexpr int kChunkBytes = kRowsPerStage * 128;            // one [16 x 32] block of a stage
+constexpr int kAChunks = kTileM / kChunk;
 constexpr int kABytes = kAChunks * kChunkBytes;             // X_hi (or X_lo) part of a stage
-constexpr int kBBytes = kBChunks * kChunkBytes;             // E_hi (or E_lo) part of a stage
-constexpr int kStageBytes = 2 * kABytes + 2 * kBBytes;
-constexpr int kSmemBytes = kStages * kStageBytes + 1024;    // + slack for 1024-byte alignment
 constexpr int kEpilogueWarps = 4;
 constexpr int kEpilogueThreads = kEpilogueWarps * 32;
 constexpr int kThreads = 64 + kEpilogueThreads;
-constexpr int kMaxAcc = 512 / kTileN - 1;                   // main accumulators beside the cross-term one
-constexpr int kStagePitch = kTileN + 4;                     // floats per row of the output staging tile
-static_assert(kTileM * kStagePitch * 4 <= kStages * kStageBytes, "output staging fits in the operand stages");
-static_assert(kTileM * kTileN * 4 <= kStages * kStageBytes, "so does the tile in the TMA store's box layout");
+
+// Sizes that follow from the tile width (classes per CTA = accumulator columns).
+template <int TILE_N>
+struct Shape {
+    static constexpr int kBChunks = TILE_N / kChunk;
+    static constexpr int kBBytes = kBChunks * kChunkBytes;              // E_hi (or E_lo) part of a stage
+    static constexpr int kStageBytes = 2 * kABytes + 2 * kBBytes;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024;     // + slack for 1024-byte alignment
+    static constexpr int kMaxAcc = 512 / TILE_N - 1;                    // main accumulators beside the cross-term one
+    static constexpr int kStagePitch = TILE_N + 4;                      // floats per row of the output staging tile
+    static_assert(kTileM * kStagePitch * 4 <= kStages * kStageBytes, "output staging fits in the operand stages");
+    static_assert(kTileM * TILE_N * 4 <= kStages * kStageBytes, "so does the tile in the TMA store's box layout");
+};
+constexpr int kWideTileMaxRows = 1024;  // 128-column tiles have three main accumulators: chains of <= 1024 / 3 rows
 
 struct GradArgs {
-    CUtensorMap x_hi, x_lo;        // [padded rows, D], boxes of 16 rows x 32, 128-byte swizzle of 32-byte pieces
-    CUtensorMap e_hi, e_lo;        // [padded rows, C]
-    float* out[DB_MAX_K];          // G_w, [D, C] row-major
-    int tma_store;                 // G_w are 16-byte aligned and C % 4 == 0: out_map[] is valid, tiles leave by TMA
-    CUtensorMap out_map[DB_MAX_K]; // G_w as [D, C], boxes of 128 rows x 32 columns, 128-byte swizzle
-    int row0[DB_MAX_K];            // first row of worker w in the split arrays (multiple of 8)
+    // The split arrays seen as [32-column chunk][row][32 floats] (the chunk stride, 128 bytes, is smaller than
+    // the row stride), 128-byte swizzle of 32-byte pieces: one box of {32, 16 rows, n chunks} fills the
+    // chunk-major tile of a stage with a single copy instruction.
+    CUtensorMap x_hi, x_lo;        // [padded rows, D], boxes of 4 chunks
+    CUtensorMap e_hi, e_lo;        // [padded rows, C], boxes of TILE_N / 32 chunks
+    // Workers in the order the CTAs take them: group g (blockIdx.z) owns slots group_begin[g] .. group_begin[g + 1])
+    int group_begin[DB_MAX_K + 1];
+    float* out[DB_MAX_K];          // G of the worker in slot z, [D, C] row-major
+    int tma_store;                 // every G is 16-byte aligned and C % 4 == 0: out_map[] is valid, tiles leave by TMA
+    CUtensorMap out_map[DB_MAX_K]; // G as [D, C], boxes of 128 rows x 32 columns, 128-byte swizzle
+    int row0[DB_MAX_K];            // first row of the worker in the split arrays (multiple of 8)
     int steps[DB_MAX_K];           // its padded row count / 8
     int D, C;
     int n_acc;                     // main accumulators in use, 1..kMaxAcc
     int* status;
+    // mean loss of the worker in slot z = (sum of row_loss[loss_row0[z] .. + loss_rows[z])) / loss_rows[z],
+    // written to loss_out[z] by the CTA with blockIdx.x == blockIdx.y == 0; row_loss == nullptr: not wanted
+    const float* row_loss;
+    float* loss_out[DB_MAX_K];
+    int loss_row0[DB_MAX_K];
+    int loss_rows[DB_MAX_K];
 };
 
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
@@ -75,6 +100,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(tc::smem_u32(bar)) : "memory");
+}
+
+// One box of a 3-D tensor map; x (elements of the contiguous dimension) must be a multiple of 4.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(tc::smem_u32(bar)) : "memory");
 }
 
 // One box from shared memory to a 2-D tensor map (rows and columns outside the tensor are not written),
@@ -108,23 +140,38 @@ __host__ __device__ constexpr uint32_t instr_desc_tf32_mn(int M, int N) {
            (static_cast<uint32_t>(M >> 4) << 24);
 }
 
-// grid: (ceil(C / 64), ceil(D / 128), workers)
+// Barrier 1 over the epilogue threads that also ANDs a predicate: the same answer in every thread.
+__device__ __forceinline__ bool epilogue_all(bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "bar.red.and.pred q, 1, %2, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(out) : "r"(static_cast<uint32_t>(pred)), "n"(kEpilogueThreads) : "memory");
+    return out != 0;
+}
+
+// grid: (ceil(C / TILE_N), ceil(D / 128), groups of workers)
+template <int TILE_N>
 __global__ void __launch_bounds__(kThreads)
 grad_tma_kernel(const __grid_constant__ GradArgs g) {
+    using S = Shape<TILE_N>;
+    constexpr int kStageBytes = S::kStageBytes, kBBytes = S::kBBytes, kStagePitch = S::kStagePitch;
     extern __shared__ unsigned char smem_raw[];
-    __shared__ __align__(8) uint64_t full_bar[kStages];
-    __shared__ __align__(8) uint64_t empty_bar[kStages];
-    __shared__ __align__(8) uint64_t done_bar;
+    __shared__ __align__(8) uint64_t full_bar[kStages];     // a stage's copies have landed
+    __shared__ __align__(8) uint64_t empty_bar[kStages];    // the products reading it have finished
+    __shared__ __align__(8) uint64_t done_bar;              // all products of the current worker have finished
+    __shared__ __align__(8) uint64_t tile_free_bar;         // its tile has left: accumulators and stages are free again
+    __shared__ __align__(8) uint64_t drain_bar;             // after a time-out: what had been issued has finished
     __shared__ uint32_t tmem_base_slot;
     __shared__ volatile int abort_flag;
 
     unsigned char* tiles = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int z = blockIdx.z;
-    const int m0 = blockIdx.y * kTileM, n0 = blockIdx.x * kTileN;
-    const int steps = g.steps[z];
-    const int loads = (steps * kStepRows + kRowsPerStage - 1) / kRowsPerStage;
+    const int z_begin = g.group_begin[blockIdx.z], z_end = g.group_begin[blockIdx.z + 1];
+    const int m0 = blockIdx.y * kTileM, n0 = blockIdx.x * TILE_N;
 
     if (tid == 0) {
         abort_flag = 0;
@@ -133,9 +180,11 @@ grad_tma_kernel(const __grid_constant__ GradArgs g) {
             tc::mbar_init(&empty_bar[s], 1);
         }
         tc::mbar_init(&done_bar, 1);
+        tc::mbar_init(&tile_free_bar, 1);
+        tc::mbar_init(&drain_bar, 1);
         tc::fence_barrier_init();
     }
-    const uint32_t tmem_cols = tc::tmem_columns((g.n_acc + 1) * kTileN);
+    const uint32_t tmem_cols = tc::tmem_columns((g.n_acc + 1) * TILE_N);
     if (warp == 1) tc::tmem_alloc(&tmem_base_slot, tmem_cols);
     tc::tc_fence_before();
     __syncthreads();
@@ -148,28 +197,27 @@ grad_tma_kernel(const __grid_constant__ GradArgs g) {
     if (warp == 0) {
         // ------------------------------------------------------------ TMA copies
         if (lane == 0) {
-            int issued = 0;
-            for (int l = 0; l < loads; ++l) {
-                const int s = l % kStages;
-                if (l >= kStages &&
-                    !tc::mbar_wait(&empty_bar[s], ((l / kStages) - 1) & 1, &abort_flag, g.status, 4))
-                    break;
-                if (abort_flag) break;
-                mbar_expect_tx(&full_bar[s], kStageBytes);
-                const uint32_t dst = tc::smem_u32(tiles + s * kStageBytes);
-                const int row = g.row0[z] + l * kRowsPerStage;
-#pragma unroll
-                for (int c = 0; c < kAChunks; ++c) {
-                    tma_load_2d(dst + c * kChunkBytes, &g.x_hi, m0 + c * kChunk, row, &full_bar[s]);
-                    tma_load_2d(dst + kABytes + c * kChunkBytes, &g.x_lo, m0 + c * kChunk, row, &full_bar[s]);
+            int issued = 0;             // stages filled so far, over all workers of the group
+            bool alive = true;
+            for (int z = z_begin; z < z_end && alive; ++z) {
+                // the previous worker's tile is staged in the operand stages until it has been stored
+                if (z > z_begin) alive = tc::mbar_wait(&tile_free_bar, (z - z_begin - 1) & 1, &abort_flag, g.status, 7);
+                const int loads = (g.steps[z] * kStepRows + kRowsPerStage - 1) / kRowsPerStage;
+                for (int l = 0; l < loads && alive; ++l) {
+                    const int s = issued % kStages;
+                    if (issued >= kStages)
+                        alive = tc::mbar_wait(&empty_bar[s], ((issued / kStages) - 1) & 1, &abort_flag, g.status, 4);
+                    if (abort_flag) alive = false;
+                    if (!alive) break;
+                    mbar_expect_tx(&full_bar[s], kStageBytes);
+                    const uint32_t dst = tc::smem_u32(tiles + s * kStageBytes);
+                    const int row = g.row0[z] + l * kRowsPerStage;
+                    tma_load_3d(dst, &g.x_hi, 0, row, m0 / kChunk, &full_bar[s]);
+                    tma_load_3d(dst + kABytes, &g.x_lo, 0, row, m0 / kChunk, &full_bar[s]);
+                    tma_load_3d(dst + 2 * kABytes, &g.e_hi, 0, row, n0 / kChunk, &full_bar[s]);
+                    tma_load_3d(dst + 2 * kABytes + kBBytes, &g.e_lo, 0, row, n0 / kChunk, &full_bar[s]);
+                    ++issued;
                 }
-#pragma unroll
-                for (int c = 0; c < kBChunks; ++c) {
-                    tma_load_2d(dst + 2 * kABytes + c * kChunkBytes, &g.e_hi, n0 + c * kChunk, row, &full_bar[s]);
-                    tma_load_2d(dst + 2 * kABytes + kBBytes + c * kChunkBytes, &g.e_lo, n0 + c * kChunk, row,
-                                &full_bar[s]);
-                }
-                issued = l + 1;
             }
             // the copies issued last write into this CTA's shared memory until they land: see them
             // complete (bounded) before this thread lets the CTA exit, whatever the other roles do
@@ -179,66 +227,96 @@ grad_tma_kernel(const __grid_constant__ GradArgs g) {
                        tc::global_ns() - t0 < tc::kWaitLimitNs) {}
             }
         }
+        // the workers' mean losses: the per-sample losses were written by the kernel before this one
+        if (g.row_loss != nullptr && blockIdx.x == 0 && blockIdx.y == 0) {
+            __syncwarp();
+            for (int z = z_begin; z < z_end; ++z) {
+                if (g.loss_out[z] == nullptr) continue;
+                const float* rl = g.row_loss + g.loss_row0[z];
+                float part = 0.0f;
+                for (int r = lane; r < g.loss_rows[z]; r += 32) part += __ldcg(rl + r);
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+                if (lane == 0) *g.loss_out[z] = part / static_cast<float>(g.loss_rows[z]);
+            }
+        }
     } else if (warp == 1) {
         // ------------------------------------------------------------ tensor-core issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = instr_desc_tf32_mn(kTileM, kTileN);
-            const uint32_t acc_cross = tmem_base + g.n_acc * kTileN;
+            constexpr uint32_t idesc = instr_desc_tf32_mn(kTileM, TILE_N);
+            const uint32_t acc_cross = tmem_base + g.n_acc * TILE_N;
             bool alive = true;
-            for (int l = 0; l < loads && alive; ++l) {
-                const int s = l % kStages;
-                alive = tc::mbar_wait(&full_bar[s], (l / kStages) & 1, &abort_flag, g.status, 5);
-                if (!alive) break;
-                tc::tc_fence_after();
-                const uint32_t st = tc::smem_u32(tiles + s * kStageBytes);
-                const int blk = l * kRowsPerStage / kAccRows;          // which 32-sample block
-                const bool blk_start = (l * kRowsPerStage) % kAccRows == 0;
-                const uint32_t acc_main = tmem_base + (blk % g.n_acc) * kTileN;
-                const int here = min(kRowsPerStage / kStepRows, steps - l * (kRowsPerStage / kStepRows));
-                for (int q = 0; q < here; ++q) {
-                    const uint32_t off = q * 1024;      // 8 rows of 128 bytes
-                    const uint64_t a_hi = smem_desc_mn_sw128(st + off);
-                    const uint64_t a_lo = smem_desc_mn_sw128(st + kABytes + off);
-                    const uint64_t b_hi = smem_desc_mn_sw128(st + 2 * kABytes + off);
-                    const uint64_t b_lo = smem_desc_mn_sw128(st + 2 * kABytes + kBBytes + off);
-                    tc::mma_tf32(acc_cross, a_lo, b_hi, idesc, (l | q) != 0);
-                    tc::mma_tf32(acc_cross, a_hi, b_lo, idesc, 1);
-                    tc::mma_tf32(acc_main, a_hi, b_hi, idesc, blk >= g.n_acc || !blk_start || q != 0);
+            int used_stages = 0;        // stages consumed so far, over all workers of the group
+            for (int z = z_begin; z < z_end && alive; ++z) {
+                // the accumulators still hold the previous worker's sums until its epilogue has read them
+                if (z > z_begin) {
+                    alive = tc::mbar_wait(&tile_free_bar, (z - z_begin - 1) & 1, &abort_flag, g.status, 9);
+                    if (!alive) break;
+                    tc::tc_fence_after();
                 }
-                tc::mma_commit(&empty_bar[s]);
+                const int steps = g.steps[z];
+                const int loads = (steps * kStepRows + kRowsPerStage - 1) / kRowsPerStage;
+                for (int l = 0; l < loads && alive; ++l) {
+                    const int s = used_stages % kStages;
+                    alive = tc::mbar_wait(&full_bar[s], (used_stages / kStages) & 1, &abort_flag, g.status, 5);
+                    if (!alive) break;
+                    tc::tc_fence_after();
+                    const uint32_t st = tc::smem_u32(tiles + s * kStageBytes);
+                    const int blk = l * kRowsPerStage / kAccRows;          // which 32-sample block
+                    const bool blk_start = (l * kRowsPerStage) % kAccRows == 0;
+                    const uint32_t acc_main = tmem_base + (blk % g.n_acc) * TILE_N;
+                    const int here = min(kRowsPerStage / kStepRows, steps - l * (kRowsPerStage / kStepRows));
+                    for (int q = 0; q < here; ++q) {
+                        const uint32_t off = q * 1024;      // 8 rows of 128 bytes
+                        const uint64_t a_hi = smem_desc_mn_sw128(st + off);
+                        const uint64_t a_lo = smem_desc_mn_sw128(st + kABytes + off);
+                        const uint64_t b_hi = smem_desc_mn_sw128(st + 2 * kABytes + off);
+                        const uint64_t b_lo = smem_desc_mn_sw128(st + 2 * kABytes + kBBytes + off);
+                        tc::mma_tf32(acc_cross, a_lo, b_hi, idesc, (l | q) != 0);
+                        tc::mma_tf32(acc_cross, a_hi, b_lo, idesc, 1);
+                        tc::mma_tf32(acc_main, a_hi, b_hi, idesc, blk >= g.n_acc || !blk_start || q != 0);
+                    }
+                    tc::mma_commit(&empty_bar[s]);
+                    ++used_stages;
+                }
+                if (alive) tc::mma_commit(&done_bar);
             }
-            tc::mma_commit(&done_bar);
             if (!alive) {
+                // a wait gave up somewhere in the CTA: see, bounded, what had been issued finish before the
+                // tensor memory is freed
+                tc::mma_commit(&drain_bar);
                 const unsigned long long t0 = tc::global_ns();
-                while (!tc::mbar_try_wait(&done_bar, 0) && tc::global_ns() - t0 < tc::kWaitLimitNs) {}
+                while (!tc::mbar_try_wait(&drain_bar, 0) && tc::global_ns() - t0 < tc::kWaitLimitNs) {}
             }
             tc::tc_fence_before();
         }
     } else {
         // ------------------------------------------------------------ epilogue
-        // the verdict is made the same for the whole warp: tcgen05.ld below is a warp-wide instruction
-        const bool alive = __all_sync(0xffffffffu, tc::mbar_wait(&done_bar, 0, &abort_flag, g.status, 6));
-        tc::tc_fence_after();
         const int et = tid - 64;                     // 0..127
         const int quarter = warp & 3;                // the tensor-memory lanes this warp may read
-        if (alive) {
-            const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+        const int row = quarter * 32 + lane;
+        float* srow = reinterpret_cast<float*>(tiles) + row * kStagePitch;
+        for (int z = z_begin; z < z_end; ++z) {
+            // the verdict is made the same for all four warps (a barrier that ANDs their predicates): what
+            // follows has warp-wide instructions and barriers among them
+            if (!epilogue_all(tc::mbar_wait(&done_bar, (z - z_begin) & 1, &abort_flag, g.status, 6))) break;
+            tc::tc_fence_after();
+            const int steps = g.steps[z];
             const int used = min(g.n_acc, (steps * kStepRows + kAccRows - 1) / kAccRows);
-            const int row = quarter * 32 + lane;
-            float* srow = reinterpret_cast<float*>(tiles) + row * kStagePitch;
 #pragma unroll 1
-            for (int c0 = 0; c0 < kTileN; c0 += 32) {
+            for (int c0 = 0; c0 < TILE_N; c0 += 32) {
                 uint32_t r[32], x[32];
                 __syncwarp();
-                tc::tmem_load32(lane_base + g.n_acc * kTileN + c0, r);
+                tc::tmem_load32(lane_base + g.n_acc * TILE_N + c0, r);
                 for (int a = used - 1; a >= 0; --a) {
-                    tc::tmem_load32(lane_base + a * kTileN + c0, x);
+                    tc::tmem_load32(lane_base + a * TILE_N + c0, x);
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
                         r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(x[j]));
                 }
                 if (g.tma_store) {
-                    // the box layout of the store: [32-column half][128 rows][128 bytes], 16-byte pieces
+                    // the box layout of the store: [32-column block][128 rows][128 bytes], 16-byte pieces
                     // permuted by the row's low three bits (which also keeps these stores conflict-free)
                     unsigned char* box = tiles + (c0 / 32) * (kTileM * 128) + row * 128;
 #pragma unroll
@@ -255,40 +333,45 @@ grad_tma_kernel(const __grid_constant__ GradArgs g) {
                 }
             }
             if (g.tma_store) tc::fence_proxy_async_smem();    // the TMA engine reads what these threads wrote
-        }
-        asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
-        if (alive && g.tma_store) {
-            if (et == 0) {
+            tc::tc_fence_before();                            // the accumulators have been read
+            asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
+            if (g.tma_store) {
+                if (et == 0) {
 #pragma unroll
-                for (int h = 0; h < kTileN / 32; ++h)
-                    if (n0 + h * 32 < g.C)
-                        tma_store_2d(&g.out_map[z], n0 + h * 32, m0, tc::smem_u32(tiles + h * (kTileM * 128)));
-                bulk_commit();
-                bulk_wait_read();      // shared memory must stay until the engine has read the tile
-            }
-        } else if (alive) {
-            // whole rows of the tile, 16 threads per row
-            const float* stage = reinterpret_cast<const float*>(tiles);
-            float* obase = g.out[z];
-            const int rows = min(kTileM, g.D - m0), cols = min(kTileN, g.C - n0);
-            constexpr int kVecPerRow = kTileN / 4;
-            constexpr int kRowsPerPass = kEpilogueThreads / kVecPerRow;
-            const int vcol = (et % kVecPerRow) * 4, rsub = et / kVecPerRow;
-            const bool vec_ok = (g.C % 4 == 0) && (reinterpret_cast<uintptr_t>(obase) % 16 == 0);
-            for (int r0 = 0; r0 < rows; r0 += kRowsPerPass) {
-                const int rr = r0 + rsub;
-                if (rr >= rows || vcol >= cols) continue;
-                const float4 val = *reinterpret_cast<const float4*>(stage + rr * kStagePitch + vcol);
-                float* dst = obase + static_cast<long long>(m0 + rr) * g.C + n0 + vcol;
-                if (vec_ok && vcol + 4 <= cols) {
-                    *reinterpret_cast<float4*>(dst) = val;
-                } else {
-                    dst[0] = val.x;
-                    if (vcol + 1 < cols) dst[1] = val.y;
-                    if (vcol + 2 < cols) dst[2] = val.z;
-                    if (vcol + 3 < cols) dst[3] = val.w;
+                    for (int h = 0; h < TILE_N / 32; ++h)
+                        if (n0 + h * 32 < g.C)
+                            tma_store_2d(&g.out_map[z], n0 + h * 32, m0, tc::smem_u32(tiles + h * (kTileM * 128)));
+                    bulk_commit();
+                    bulk_wait_read();      // shared memory must stay until the engine has read the tile
                 }
+            } else {
+                // whole rows of the tile, TILE_N / 4 threads per row
+                const float* stage = reinterpret_cast<const float*>(tiles);
+                float* obase = g.out[z];
+                const int rows = min(kTileM, g.D - m0), cols = min(TILE_N, g.C - n0);
+                constexpr int kVecPerRow = TILE_N / 4;
+                constexpr int kRowsPerPass = kEpilogueThreads / kVecPerRow;
+                const int vcol = (et % kVecPerRow) * 4, rsub = et / kVecPerRow;
+                const bool vec_ok = (g.C % 4 == 0) && (reinterpret_cast<uintptr_t>(obase) % 16 == 0);
+                for (int r0 = 0; r0 < rows; r0 += kRowsPerPass) {
+                    const int rr = r0 + rsub;
+                    if (rr >= rows || vcol >= cols) continue;
+                    const float4 val = *reinterpret_cast<const float4*>(stage + rr * kStagePitch + vcol);
+                    float* dst = obase + static_cast<long long>(m0 + rr) * g.C + n0 + vcol;
+                    if (vec_ok && vcol + 4 <= cols) {
+                        *reinterpret_cast<float4*>(dst) = val;
+                    } else {
+                        dst[0] = val.x;
+                        if (vcol + 1 < cols) dst[1] = val.y;
+                        if (vcol + 2 < cols) dst[2] = val.z;
+                        if (vcol + 3 < cols) dst[3] = val.w;
+                    }
+                }
+                // every thread has read its part of the staging tile before the stages are handed back
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
             }
+            // stages and accumulators may be reused by the next worker of the group
+            if (et == 0 && z + 1 < z_end) tc::mbar_arrive(&tile_free_bar);
         }
         tc::tc_fence_before();
     }

@@ -55,6 +55,7 @@ struct LogitArgs {
     int k_per_split;               // multiple of 32
     int n_acc;                     // main accumulators, (n_acc + 1) * N_TILE <= 512
     int* status;
+    int clear_status;              // non-zero: the first CTA zeroes *status before any wait can set it
 };
 
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
@@ -132,6 +133,8 @@ logits_tma_kernel(const __grid_constant__ LogitArgs g) {
     const uint32_t tmem_base = tmem_base_slot;
     tc::griddep_launch_dependents();
     tc::griddep_wait();
+    // a time-out needs seconds, this store comes microseconds after the launch: no wait can have given up yet
+    if (g.clear_status && tid == 0 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) *g.status = 0;
 
     if (warp == kSplitWarps + 1) {
         // ------------------------------------------------------------ TMA copies: lanes 0-3 a W chunk each, lane 4 X

@@ -3,13 +3,16 @@
 // the model on which Eq. 2's batch-proportional weights are checked against
 // the gradient of the concatenated global batch (Section 3.1).
 //
-// A memset node (status word and tickets) and three launches on the caller's stream:
+// Three launches on the caller's stream, each scheduled under its predecessor (programmatic
+// dependent launch) and waiting for it before it reads its output:
 //   1. logits: split over the feature dimension D so that a worker with a
 //      handful of rows still fills the GPU; partial sums go to the workspace;
+//      its first CTA also zeroes the status word of the call;
 //   2. softmax: one CTA per sample folds the partials in split order, applies
 //      the max-subtracted softmax, subtracts the one-hot label, scales by 1/b_i;
-//      the last CTA of a worker also folds the per-sample losses into the mean;
-//   3. gradient: G = X^T E, reduction depth b_i.
+//   3. gradient: G = X^T E, reduction depth b_i; one CTA per worker also folds
+//      the per-sample losses into the worker's mean loss.
+// (The FFMA path keeps a memset node for its status word and loss ticket.)
 // The two contractions run on the tensor cores (tcgen05, three TF32 products per
 // fp32 product), fed by TMA: the logits read W and X where the caller left them
 // (tc_logits.cuh; unaligned inputs go through the register-converting contraction of
@@ -207,6 +210,9 @@ softmax_residual_kernel(const float* __restrict__ partials, int splits, long lon
         el = so.e_lo + static_cast<long long>(ip) * so.e_pitch;
         float* xh = so.x_hi + static_cast<long long>(ip) * so.x_pitch;
         float* xl = so.x_lo + static_cast<long long>(ip) * so.x_pitch;
+        // the columns between C (D) and the pitch are copied with the rest of their 32-column chunk: zeros
+        for (int c = C + threadIdx.x; c < so.e_pitch; c += kThreads) { eh[c] = 0.0f; el[c] = 0.0f; }
+        for (int d = so.D + threadIdx.x; d < so.x_pitch; d += kThreads) { xh[d] = 0.0f; xl[d] = 0.0f; }
         if (r >= groups.off[w + 1] - groups.off[w]) {
             // padding row: zeros in all four arrays (the workspace may hold anything, NaN included)
             for (int c = threadIdx.x; c < C; c += kThreads) { eh[c] = 0.0f; el[c] = 0.0f; }
@@ -457,7 +463,7 @@ bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0;
 // defined below, beside the grouped entry point
 db_status launch_logits_tma(const float* X, long long x_pitch, const float* W, long long w_pitch, float* partials,
                             long long o_split, long long o_n, int rows, int D, int C, int k_per_split, int n_tile,
-                            int* status, cudaStream_t stream);
+                            int* status, bool first_of_call, cudaStream_t stream);
 size_t grouped_workspace_total(long long rows, int K, int D, int C);
 db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, const int32_t* offsets, int K, int D,
                              int C, float* const* G, float* losses, void* workspace, cudaStream_t stream);
@@ -479,7 +485,7 @@ extern "C" db_status db_contract_f32(const float* A, int64_t a_row, int64_t a_k,
     const int k_round = K > 0 ? (K + tc::kBlockK - 1) / tc::kBlockK * tc::kBlockK : tc::kBlockK;
     // A contiguous along m, B along k, out along m: the layout of the logits, operands by TMA
     if (K > 0 && a_row == 1 && a_k % 4 == 0 && aligned16(A) && b_k == 1 && b_row % 4 == 0 && aligned16(B) && o_m == 1)
-        return launch_logits_tma(B, b_row, A, a_k, out, 0, o_n, N, K, M, k_round, n_tile, status,
+        return launch_logits_tma(B, b_row, A, a_k, out, 0, o_n, N, K, M, k_round, n_tile, status, false,
                                  static_cast<cudaStream_t>(cuda_stream));
     tc::GemmArgs a{};
     a.A = A; a.a_row = a_row; a.a_k = a_k;
@@ -649,12 +655,39 @@ db_status make_operand_map(CUtensorMap* map, const float* base, long long rows, 
     return DB_OK;
 }
 
+// Tensor map of a row-major fp32 array [rows, pitch] (pitch a multiple of 32 floats) seen as
+// [pitch / 32 chunks][rows][32 floats]: the chunk stride (128 bytes) is smaller than the row stride, which
+// the encoder accepts.  A box of {32, box_rows, box_chunks} lands in shared memory chunk-major, each
+// chunk a [box_rows x 128 bytes] block with the 128-byte swizzle of 32-byte pieces; rows beyond `rows`
+// read as zero.  Every column of the pitch must hold finite data or belong to an output that is never
+// stored.
+db_status make_chunked_map(CUtensorMap* map, const float* base, long long rows, long long pitch, int box_rows,
+                           int box_chunks) {
+    EncodeTiledFn enc = encode_tiled();
+    if (!enc) {
+        record_message("cuTensorMapEncodeTiled is not available from this driver");
+        return DB_ERR_CUDA;
+    }
+    const cuuint64_t dims[3] = {32, static_cast<cuuint64_t>(rows), static_cast<cuuint64_t>(pitch / 32)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(pitch) * sizeof(float), 128};
+    const cuuint32_t box[3] = {32, static_cast<cuuint32_t>(box_rows), static_cast<cuuint32_t>(box_chunks)};
+    const cuuint32_t elem[3] = {1, 1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, elem,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        record_message("cuTensorMapEncodeTiled rejected the chunked layout of a gradient operand");
+        return DB_ERR_CUDA;
+    }
+    return DB_OK;
+}
+
 // out(n, c) = sum_d X(n, d) W(d, c) with both operands copied by TMA from where the caller left them
 // (the logits; also db_contract_f32 for operands laid out that way).  Needs 16-byte aligned W and X and
 // row pitches that are multiples of 4 floats; out(n, c) lands at out[split * o_split + n * o_n + c].
 db_status launch_logits_tma(const float* X, long long x_pitch, const float* W, long long w_pitch, float* partials,
                             long long o_split, long long o_n, int rows, int D, int C, int k_per_split, int n_tile,
-                            int* status, cudaStream_t stream) {
+                            int* status, bool first_of_call, cudaStream_t stream) {
     tcl::LogitArgs a{};
     db_status st;
     if ((st = make_operand_map(&a.w, W, D, C, w_pitch, tcl::kBlockK, true)) != DB_OK) return st;
@@ -662,6 +695,7 @@ db_status launch_logits_tma(const float* X, long long x_pitch, const float* W, l
     a.o_n = o_n;
     a.out = partials; a.o_split = o_split; a.rows = rows; a.D = D; a.C = C; a.k_per_split = k_per_split;
     a.status = status;
+    a.clear_status = first_of_call ? 1 : 0;
     // one main accumulator per four reduction blocks (chains of 16 additions), within 512 columns
     const int blocks = k_per_split / tcl::kBlockK;
     a.n_acc = std::min(std::max((blocks + 3) / 4, 1), 512 / n_tile - 1);
@@ -675,7 +709,8 @@ db_status launch_logits_tma(const float* X, long long x_pitch, const float* W, l
         default: fn = tcl::logits_tma_kernel<128>; smem = tcl::Smem<128>::kBytes; break;
     }
     DB_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    OverlappedLaunch OL(grid, dim3(tcl::kThreads), smem, stream, false);
+    // as the first kernel of a worker-gradient call it may be scheduled under whatever precedes the call
+    OverlappedLaunch OL(grid, dim3(tcl::kThreads), smem, stream, first_of_call);
     DB_CUDA_TRY(cudaLaunchKernelEx(&OL.cfg, fn, a));
     DB_CUDA_TRY(cudaGetLastError());
     return DB_OK;
@@ -688,7 +723,6 @@ db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, c
     const GroupedLayout L = grouped_layout(rows, K, D, C);
     char* base = static_cast<char*>(workspace);
     int* status = reinterpret_cast<int*>(base);
-    unsigned int* tickets = reinterpret_cast<unsigned int*>(base + kStatusBytes);
     char* cur = base + L.header_bytes;
     float* partials = reinterpret_cast<float*>(cur); cur += L.partial_bytes;
     float* E = reinterpret_cast<float*>(cur); cur += L.e_bytes;
@@ -706,26 +740,65 @@ db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, c
     for (int w = 0; w < K; ++w) rg.poff[w + 1] = rg.poff[w] + static_cast<int>(round_up(offsets[w + 1] - offsets[w], 8));
     const long long rows_p = rg.poff[K];
 
+    // Tile width of the gradient kernel: 128 classes while three main accumulators keep the chains short.
+    int max_rows = 0;
+    for (int w = 0; w < K; ++w) max_rows = std::max(max_rows, rg.poff[w + 1] - rg.poff[w]);
+    const bool wide = max_rows <= tcg::kWideTileMaxRows;
+    const int tile_n = wide ? 128 : 64;
+    const int max_acc = wide ? tcg::Shape<128>::kMaxAcc : tcg::Shape<64>::kMaxAcc;
+    const int grad_smem = wide ? tcg::Shape<128>::kSmemBytes : tcg::Shape<64>::kSmemBytes;
+    void (*grad_fn)(const tcg::GradArgs) = wide ? tcg::grad_tma_kernel<128> : tcg::grad_tma_kernel<64>;
+
     tcg::GradArgs ga{};
     db_status st;
-    if ((st = make_operand_map(&ga.x_hi, x_hi, rows_p, D, L.x_pitch, tcg::kRowsPerStage, true)) != DB_OK) return st;
-    if ((st = make_operand_map(&ga.x_lo, x_lo, rows_p, D, L.x_pitch, tcg::kRowsPerStage, true)) != DB_OK) return st;
-    if ((st = make_operand_map(&ga.e_hi, e_hi, rows_p, C, L.e_pitch, tcg::kRowsPerStage, true)) != DB_OK) return st;
-    if ((st = make_operand_map(&ga.e_lo, e_lo, rows_p, C, L.e_pitch, tcg::kRowsPerStage, true)) != DB_OK) return st;
+    if ((st = make_chunked_map(&ga.x_hi, x_hi, rows_p, L.x_pitch, tcg::kRowsPerStage, tcg::kAChunks)) != DB_OK) return st;
+    if ((st = make_chunked_map(&ga.x_lo, x_lo, rows_p, L.x_pitch, tcg::kRowsPerStage, tcg::kAChunks)) != DB_OK) return st;
+    if ((st = make_chunked_map(&ga.e_hi, e_hi, rows_p, L.e_pitch, tcg::kRowsPerStage, tile_n / tcg::kChunk)) != DB_OK) return st;
+    if ((st = make_chunked_map(&ga.e_lo, e_lo, rows_p, L.e_pitch, tcg::kRowsPerStage, tile_n / tcg::kChunk)) != DB_OK) return st;
+    // one main accumulator per four 32-sample blocks (chains of 16 additions), within the 512 columns
+    const int max_blocks = (max_rows + tcg::kAccRows - 1) / tcg::kAccRows;
+    ga.n_acc = std::min(std::max((max_blocks + 3) / 4, 1), max_acc);
 
-    // largest batches first: their CTAs run longest and should not form the tail of the grid
+    // Groups of workers: as many as keep the whole grid resident (tiles x groups <= CTA slots of the GPU),
+    // at most one per worker; the workers are dealt largest first, each to the group with the fewest rows.
+    DB_CUDA_TRY(cudaFuncSetAttribute(grad_fn, cudaFuncAttributeMaxDynamicSharedMemorySize, grad_smem));
+    static int resident[2] = {0, 0};           // CTAs per SM that the shared memory allows, per tile width
+    int per_sm = resident[wide ? 1 : 0];
+    if (per_sm == 0) {
+        DB_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, grad_fn, tcg::kThreads, grad_smem));
+        resident[wide ? 1 : 0] = per_sm;        // every thread would store the same value
+    }
+    per_sm = std::max(1, std::min(per_sm, 512 / static_cast<int>(tc::tmem_columns((ga.n_acc + 1) * tile_n))));
+    const long long grad_tiles = static_cast<long long>((C + tile_n - 1) / tile_n) * ((D + tcg::kTileM - 1) / tcg::kTileM);
+    const long long slots = static_cast<long long>(sm_count()) * per_sm;
+    const int groups = static_cast<int>(std::max(1LL, std::min<long long>(K, slots / grad_tiles)));
     int order[DB_MAX_K];
     for (int w = 0; w < K; ++w) order[w] = w;
     std::stable_sort(order, order + K, [&](int u, int v) {
         return offsets[u + 1] - offsets[u] > offsets[v + 1] - offsets[v];
     });
-    int max_steps = 1;
-    for (int z = 0; z < K; ++z) {
-        const int w = order[z];
+    int group_of[DB_MAX_K];
+    long long load[DB_MAX_K] = {0};
+    int count[DB_MAX_K] = {0};
+    for (int i = 0; i < K; ++i) {
+        int best = 0;
+        for (int gi = 1; gi < groups; ++gi)
+            if (load[gi] < load[best]) best = gi;
+        group_of[i] = best;
+        load[best] += rg.poff[order[i] + 1] - rg.poff[order[i]];
+        ++count[best];
+    }
+    ga.group_begin[0] = 0;
+    for (int gi = 0; gi < groups; ++gi) ga.group_begin[gi + 1] = ga.group_begin[gi] + count[gi];
+    int cursor[DB_MAX_K];
+    for (int gi = 0; gi < groups; ++gi) cursor[gi] = ga.group_begin[gi];
+    int slot_worker[DB_MAX_K];     // the worker a CTA slot belongs to
+    for (int i = 0; i < K; ++i) {
+        const int w = order[i], z = cursor[group_of[i]]++;
+        slot_worker[z] = w;
         ga.out[z] = G[w];
         ga.row0[z] = rg.poff[w];
         ga.steps[z] = (rg.poff[w + 1] - rg.poff[w]) / tcg::kStepRows;
-        max_steps = std::max(max_steps, ga.steps[z]);
     }
     // the tiles leave by TMA when every G_w allows it (16-byte aligned, rows a multiple of 16 bytes)
     ga.tma_store = C % 4 == 0;
@@ -733,14 +806,14 @@ db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, c
     for (int z = 0; z < K && ga.tma_store; ++z)
         if ((st = make_operand_map(&ga.out_map[z], ga.out[z], D, C, C, tcg::kTileM, false)) != DB_OK) return st;
 
-    // nothing has been enqueued up to here
-    DB_CUDA_TRY(cudaMemsetAsync(base, 0, L.header_bytes, stream));
-
+    // Nothing has been enqueued up to here.  The status word is zeroed by the first CTA of the logits
+    // kernel and the mean losses are folded by the gradient kernel, so the call is three launches and
+    // nothing else.
     // 1. logits of every row, transposed orientation, split over D; operands by TMA where their
     //    alignment allows it, else through the register-converting contraction
     if (aligned16(W) && aligned16(X) && C % 4 == 0 && D % 4 == 0) {
         st = launch_logits_tma(X, D, W, C, partials, rc, C, static_cast<int>(rows), D, C, L.k_per_split, L.n_tile,
-                               status, stream);
+                               status, true, stream);
         if (st != DB_OK) return st;
     } else {
         tc::GemmArgs a{};
@@ -748,6 +821,7 @@ db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, c
         a.B = X; a.b_row = D; a.b_k = 1;          // B(n = sample, k = feature) = X[n, k]
         a.out = partials; a.o_m = 1; a.o_n = C; a.o_split = rc;   // Z[n, m], one slab per split
         a.M = C; a.N = static_cast<int>(rows); a.K = D; a.k_per_split = L.k_per_split; a.status = status;
+        a.clear_status = 1;
         st = launch_tc_gemm(a, L.n_tile, stream);
         if (st != DB_OK) return st;
     }
@@ -757,21 +831,23 @@ db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, c
         so.e_hi = e_hi; so.e_lo = e_lo; so.e_pitch = L.e_pitch;
         so.X = X; so.x_hi = x_hi; so.x_lo = x_lo; so.x_pitch = L.x_pitch; so.D = D;
         so.x_vec = (D % 4 == 0) && aligned16(X);
-        st = launch_softmax(partials, L.splits, rc, y, E, row_loss, rg, static_cast<int>(rows), C, tickets, losses,
+        st = launch_softmax(partials, L.splits, rc, y, E, row_loss, rg, static_cast<int>(rows), C, nullptr, nullptr,
                             stream, true, &so);
         if (st != DB_OK) return st;
     }
     // 3. one gradient per worker: G_w = X_w^T E_w, reduction over that worker's rows only
     {
         ga.D = D; ga.C = C; ga.status = status;
-        // one main accumulator per four 32-sample blocks (chains of 16 additions), within the 512 columns
-        const int blocks = (max_steps * tcg::kStepRows + tcg::kAccRows - 1) / tcg::kAccRows;
-        ga.n_acc = std::min(std::max((blocks + 3) / 4, 1), tcg::kMaxAcc);
-        DB_CUDA_TRY(cudaFuncSetAttribute(tcg::grad_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         tcg::kSmemBytes));
-        dim3 grid((C + tcg::kTileN - 1) / tcg::kTileN, (D + tcg::kTileM - 1) / tcg::kTileM, K);
-        OverlappedLaunch OL(grid, dim3(tcg::kThreads), tcg::kSmemBytes, stream, true);
-        DB_CUDA_TRY(cudaLaunchKernelEx(&OL.cfg, tcg::grad_tma_kernel, ga));
+        ga.row_loss = losses ? row_loss : nullptr;
+        for (int z = 0; z < K && losses; ++z) {
+            const int w = slot_worker[z];
+            ga.loss_out[z] = losses + w;
+            ga.loss_row0[z] = offsets[w];
+            ga.loss_rows[z] = offsets[w + 1] - offsets[w];
+        }
+        dim3 grid((C + tile_n - 1) / tile_n, (D + tcg::kTileM - 1) / tcg::kTileM, groups);
+        OverlappedLaunch OL(grid, dim3(tcg::kThreads), grad_smem, stream, true);
+        DB_CUDA_TRY(cudaLaunchKernelEx(&OL.cfg, grad_fn, ga));
         DB_CUDA_TRY(cudaGetLastError());
     }
     return DB_OK;

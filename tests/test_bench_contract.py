@@ -18,6 +18,8 @@ def test_reference_arm_prints_one_contract_line():
     assert d["steps"] == 2 and d["n_gpus"] == 1 and d["value"] > 0 and d["vs_baseline"] is None
     assert d["config"]["workload"].startswith("resnet50") and "model" not in d["config"]
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1
+    one = d["cpu_baseline"]["single_thread"]
+    assert one["cores"] == 1 and one["unit"] == "GB/s" and one["value"] > 0
     assert d["e2e"] == {"value": d["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
 
 
@@ -37,3 +39,11 @@ def test_byte_formula_and_workloads():
     assert bench.bert_base_workload().bytes_per_step == 16 * 109_482_240 * 2 + 16 * 109_482_240
     pts = bench.sweep_workloads()
     assert len(pts) == 25 and max(w.K * w.N for w in pts) == 1 << 33
+
+
+def test_reference_arm_follows_the_workload():
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
+                          "--warmup", "1", "--workload", "small"], capture_output=True, text=True, timeout=600, cwd=ROOT)
+    assert out.returncode == 0, out.stderr
+    d = json.loads(out.stdout.strip().splitlines()[-1])
+    assert d["config"]["workload"].startswith("small") and d["config"]["K"] == 3 and d["config"]["N"] == 1 << 20

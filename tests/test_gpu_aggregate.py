@@ -160,6 +160,29 @@ def test_norm_of_ones_is_exactly_N():
     assert float(sq.item()) == float(N)
 
 
+def test_overlapping_steps_on_two_streams_keep_their_norms_apart():
+    """Two streams run norm-carrying steps at the same time, each with its own workspace.  Every norm
+    must be its own problem's."""
+    K, calls = 2, 300
+    sizes = (300_001, 777_777)
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    state = []
+    for i, N in enumerate(sizes):
+        g = [torch.full((N,), float(i + 1), device=DEV) for _ in range(K)]
+        state.append((g, torch.zeros(N, device=DEV), torch.zeros(N, device=DEV),
+                      torch.zeros(calls, dtype=torch.float64, device=DEV), _workspace(K, N)))
+    torch.cuda.synchronize()
+    for c in range(calls):
+        for i, s in enumerate(streams):
+            g, p, v, sq, ws = state[i]
+            binding.aggregate_update(g, [3, 5], p, v, 0.0, 0.0, sq[c:c + 1], ws, s)
+    torch.cuda.synchronize()
+    for i, N in enumerate(sizes):
+        want = float(N) * (i + 1) ** 2
+        got = state[i][3].cpu().numpy()
+        assert (got == want).all(), (i, got[got != want][:5], want)
+
+
 def test_runs_are_bit_identical_and_norm_flag_does_not_change_the_update():
     N, K = 3_000_017, 8
     g = inputs.worker_gradients(K, N, 1e-3, 90, device=DEV)
