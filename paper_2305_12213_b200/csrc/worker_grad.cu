@@ -21,10 +21,6 @@
 // shared-memory tiles is kept as the accuracy reference and for very large b_i.
 #include <algorithm>
 #include <cstdint>
-#include <functional>
-#include <queue>
-#include <utility>
-#include <vector>
 
 #include "common.h"
 #include "tc_gemm.cuh"
@@ -744,25 +740,14 @@ db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, c
     for (int w = 0; w < K; ++w) rg.poff[w + 1] = rg.poff[w] + static_cast<int>(round_up(offsets[w + 1] - offsets[w], 8));
     const long long rows_p = rg.poff[K];
 
-    // Shape of the gradient kernel: the widest tile and the most accumulator sets whose main accumulators
-    // still keep every chain of truncating tensor-memory additions short (one accumulator per four
-    // 32-sample blocks, i.e. chains of 16 additions, where the 512 columns allow it).
+    // Tile width of the gradient kernel: 128 classes while three main accumulators keep the chains short.
     int max_rows = 0;
     for (int w = 0; w < K; ++w) max_rows = std::max(max_rows, rg.poff[w + 1] - rg.poff[w]);
-    const int max_blocks = (max_rows + tcg::kAccRows - 1) / tcg::kAccRows;
-    const int want_acc = std::max((max_blocks + 3) / 4, 1);
-    int tile_n, max_acc, grad_smem;
-    void (*grad_fn)(const tcg::GradArgs);
-    if (want_acc <= tcg::Shape<128, 2>::kMaxAcc) {
-        tile_n = 128; max_acc = tcg::Shape<128, 2>::kMaxAcc; grad_smem = tcg::Shape<128, 2>::kSmemBytes;
-        grad_fn = tcg::grad_tma_kernel<128, 2>;
-    } else if (want_acc <= tcg::Shape<64, 2>::kMaxAcc) {
-        tile_n = 64; max_acc = tcg::Shape<64, 2>::kMaxAcc; grad_smem = tcg::Shape<64, 2>::kSmemBytes;
-        grad_fn = tcg::grad_tma_kernel<64, 2>;
-    } else {
-        tile_n = 64; max_acc = tcg::Shape<64, 1>::kMaxAcc; grad_smem = tcg::Shape<64, 1>::kSmemBytes;
-        grad_fn = tcg::grad_tma_kernel<64, 1>;
-    }
+    const bool wide = max_rows <= tcg::kWideTileMaxRows;
+    const int tile_n = wide ? 128 : 64;
+    const int max_acc = wide ? tcg::Shape<128>::kMaxAcc : tcg::Shape<64>::kMaxAcc;
+    const int grad_smem = wide ? tcg::Shape<128>::kSmemBytes : tcg::Shape<64>::kSmemBytes;
+    void (*grad_fn)(const tcg::GradArgs) = wide ? tcg::grad_tma_kernel<128> : tcg::grad_tma_kernel<64>;
 
     tcg::GradArgs ga{};
     db_status st;
@@ -770,9 +755,11 @@ db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, c
     if ((st = make_chunked_map(&ga.x_lo, x_lo, rows_p, L.x_pitch, tcg::kRowsPerStage, tcg::kAChunks)) != DB_OK) return st;
     if ((st = make_chunked_map(&ga.e_hi, e_hi, rows_p, L.e_pitch, tcg::kRowsPerStage, tile_n / tcg::kChunk)) != DB_OK) return st;
     if ((st = make_chunked_map(&ga.e_lo, e_lo, rows_p, L.e_pitch, tcg::kRowsPerStage, tile_n / tcg::kChunk)) != DB_OK) return st;
-    ga.n_acc = std::min(want_acc, max_acc);
+    // one main accumulator per four 32-sample blocks (chains of 16 additions), within the 512 columns
+    const int max_blocks = (max_rows + tcg::kAccRows - 1) / tcg::kAccRows;
+    ga.n_acc = std::min(std::max((max_blocks + 3) / 4, 1), max_acc);
 
-    // Slots: the workers by falling row count.  Items: every tile of every slot, in that order.
+    // largest batches first: their CTAs run longest and should not form the tail of the grid
     int order[DB_MAX_K];
     for (int w = 0; w < K; ++w) order[w] = w;
     std::stable_sort(order, order + K, [&](int u, int v) {
@@ -783,39 +770,6 @@ db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, c
         ga.out[z] = G[w];
         ga.row0[z] = rg.poff[w];
         ga.steps[z] = (rg.poff[w + 1] - rg.poff[w]) / tcg::kStepRows;
-    }
-    ga.K = K;
-    ga.tiles_x = (C + tile_n - 1) / tile_n;
-    const long long tiles_ll = static_cast<long long>(ga.tiles_x) * ((D + tcg::kTileM - 1) / tcg::kTileM);
-    const long long n_items = tiles_ll * K;
-    if (n_items > 0x7fffffffLL) return DB_ERR_ARG;
-    ga.tiles = static_cast<int>(tiles_ll);
-    ga.n_items = static_cast<int>(n_items);
-    const int grad_ctas = static_cast<int>(std::min<long long>(n_items, sm_count()));
-    // The item table: items dealt in order (most rows first), each to the CTA with the least work so far;
-    // an item costs its rows plus a constant for draining and storing its tile.
-    ga.use_table = grad_ctas <= tcg::kMaxCtas && n_items <= 65535 &&
-                   n_items <= static_cast<long long>(grad_ctas) * tcg::kMaxItemsPerCta;
-    if (ga.use_table) {
-        constexpr long long kItemOverheadRows = 64;
-        using Slot = std::pair<long long, int>;                  // (work so far, CTA): least work first, then lowest CTA
-        std::priority_queue<Slot, std::vector<Slot>, std::greater<Slot>> least;
-        for (int c = 0; c < grad_ctas; ++c) least.push({0, c});
-        for (int i = 0; i < ga.n_items && ga.use_table; ++i) {
-            std::vector<Slot> full;                              // CTAs whose row of the table is full
-            Slot top = least.top();
-            least.pop();
-            while (ga.item_count[top.second] >= tcg::kMaxItemsPerCta && !least.empty()) {
-                full.push_back(top);
-                top = least.top();
-                least.pop();
-            }
-            if (ga.item_count[top.second] >= tcg::kMaxItemsPerCta) { ga.use_table = 0; break; }
-            ga.item_table[top.second][ga.item_count[top.second]++] = static_cast<unsigned short>(i);
-            top.first += ga.steps[i / ga.tiles] * tcg::kStepRows + kItemOverheadRows;
-            least.push(top);
-            for (const Slot& f : full) least.push(f);
-        }
     }
     // the tiles leave by TMA when every G_w allows it (16-byte aligned, rows a multiple of 16 bytes)
     ga.tma_store = C % 4 == 0;
@@ -863,7 +817,8 @@ db_status worker_grad_tensor(const float* X, const int32_t* y, const float* W, c
             ga.loss_rows[z] = offsets[w + 1] - offsets[w];
         }
         DB_CUDA_TRY(cudaFuncSetAttribute(grad_fn, cudaFuncAttributeMaxDynamicSharedMemorySize, grad_smem));
-        OverlappedLaunch OL(dim3(grad_ctas), dim3(tcg::kThreads), grad_smem, stream, true);
+        dim3 grid((C + tile_n - 1) / tile_n, (D + tcg::kTileM - 1) / tcg::kTileM, K);
+        OverlappedLaunch OL(grid, dim3(tcg::kThreads), grad_smem, stream, true);
         DB_CUDA_TRY(cudaLaunchKernelEx(&OL.cfg, grad_fn, ga));
         DB_CUDA_TRY(cudaGetLastError());
     }
