@@ -176,7 +176,8 @@ grad_tma_kernel(const __grid_constant__ GradArgs g) {
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int z = blockIdx.z;
-    const int steps = g.steps[z];
+    // read from the parameter block before the wait for the previous kernel, not after it
+    const int steps = g.steps[z], first_row = g.row0[z];
     const int loads = (steps * kStepRows + kRowsPerStage - 1) / kRowsPerStage;
     const int m0 = blockIdx.y * kTileM, n0 = blockIdx.x * TILE_N;
 
@@ -216,7 +217,7 @@ grad_tma_kernel(const __grid_constant__ GradArgs g) {
                 if (abort_flag) break;
                 mbar_expect_tx(&full_bar[s], kStageBytes);
                 const uint32_t dst = tc::smem_u32(tiles + s * kStageBytes);
-                const int row = g.row0[z] + l * kRowsPerStage;
+                const int row = first_row + l * kRowsPerStage;
                 tma_load_3d(dst, &g.x_hi, 0, row, m0 / kChunk, &full_bar[s]);
                 tma_load_3d(dst + kABytes, &g.x_lo, 0, row, m0 / kChunk, &full_bar[s]);
                 tma_load_3d(dst + 2 * kABytes, &g.e_hi, 0, row, n0 / kChunk, &full_bar[s]);

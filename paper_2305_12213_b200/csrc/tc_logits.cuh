@@ -17,9 +17,11 @@
 // 320 threads: warps 0-7 derive the lo halves and later drain the accumulators, warp 8 owns tensor
 // memory and (one lane) issues the products, warp 9 issues the copies: five lanes, one box each, in
 // the same instruction (measured: a further box costs about half as much that way as from the same
-// thread, and an iteration of the copy loop costs 0.3 us before its first box).  Before
-// its first copy that warp asks the L2 to prefetch every box of the CTA's share of W, so that the
-// ring of three stages meets L2 latencies, not DRAM's.  Every wait is bounded as in tc_gemm.cuh.
+// thread, and an iteration of the copy loop costs 0.3 us before its first box).  While the
+// first stage is on its way, the threads of warps 0-7 ask the L2 to prefetch every later box of the
+// CTA's share of W, one box each, so that the ring of three stages meets L2 latencies, not DRAM's
+// (issued in a row by the copying warp these requests delayed its first copy by 1.6 us).
+// Every wait is bounded as in tc_gemm.cuh.
 #pragma once
 #include <cuda.h>
 
@@ -124,6 +126,8 @@ logits_tma_kernel(const __grid_constant__ LogitArgs g) {
         }
         tc::mbar_init(&done_bar, 1);
         tc::fence_barrier_init();
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&g.w)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&g.x)) : "memory");
     }
     const uint32_t tmem_cols = tc::tmem_columns((g.n_acc + 1) * N_TILE);
     if (warp == kSplitWarps) tc::tmem_alloc(&tmem_base_slot, tmem_cols);
@@ -141,10 +145,6 @@ logits_tma_kernel(const __grid_constant__ LogitArgs g) {
         const bool is_w = lane < kAChunks;
         const CUtensorMap* map = is_w ? &g.w : &g.x;
         const uint32_t box_off = is_w ? lane * kAChunkBytes : 2 * kABytes;
-        if (is_w) {
-            for (int kb = 0; kb < nkb; ++kb) tma_prefetch_2d(&g.w, m0 + lane * 32, k_begin + kb * kBlockK);
-        }
-        __syncwarp();
         int issued = 0;
         for (int kb = 0; kb < nkb; ++kb) {
             const int s = kb % kStages;
@@ -210,6 +210,11 @@ logits_tma_kernel(const __grid_constant__ LogitArgs g) {
         }
     } else {
         // ------------------------------------------------------------ lo halves, then the epilogue
+        // First, while the first stage is on its way: ask the L2 to fetch the boxes of W that the later
+        // stages will copy, one box per thread (a TMA instruction costs its thread 0.2 - 0.4 us, measured, so
+        // they are issued side by side here rather than in a row by the copying warp).
+        if (tid >= kAChunks && tid < nkb * kAChunks)
+            tma_prefetch_2d(&g.w, m0 + (tid % kAChunks) * 32, k_begin + (tid / kAChunks) * kBlockK);
         bool alive = true;
         for (int kb = 0; kb < nkb; ++kb) {
             const int s = kb % kStages;
