@@ -494,6 +494,65 @@ def measure_softmax(args, dev, rank, world):
     }
 
 
+def measure_sharded(args, dev, rank, world):
+    """Opt-in: the ResNet-50-shaped step with one parameter server per GPU (sharded.ShardedServer): every rank
+    hosts K / world of the workers' gradient buffers and owns 1 / world of the parameters; per step a barrier,
+    the fused kernel on the slice (peer loads for the other ranks' workers), an all-gather of the parameters and
+    an all-reduce of the norm.  Strong scaling: the job is one model, whatever the number of GPUs."""
+    from paper_2305_12213_b200 import binding, sharded
+    wl = resnet50_workload()
+    if wl.K % world:
+        raise SystemExit(f"--mode sharded: {wl.K} workers do not divide over {world} ranks")
+    k_local = wl.K // world
+    local = inputs.worker_gradients(k_local, wl.N, wl.grad_std, 2000 + 100 * rank, device=dev, dtype=wl.grad_dtype)
+    p0 = inputs.normal(wl.N, PARAM_STD, 2500, dev)
+    server = sharded.ShardedServer(local, p0)
+    b = list(wl.b0)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        nonlocal b
+        b = binding.controller_step(b, wl.throughputs, wl.kp)
+        server.step(b, wl.lr, wl.mu)
+
+    warmup = max(3, args.warmup)
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(dev.index)
+    replicas.barrier(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with sampler:
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+    replicas.barrier(dev)
+    ms = replicas.max_over_ranks(e0.elapsed_time(e1), dev)
+    bytes_step = wl.bytes_per_step                       # the whole job's step, not per rank
+    sq = float(server.sqnorm.item())
+    assert np.isfinite(sq) and sq > 0
+    peak, peak_kind = measured_peak()
+    achieved = bytes_step / world / (ms / args.steps * 1e-3) / 1e9
+    return {
+        "metric": f"{METRIC} [one parameter server per GPU]", "value": bytes_step * args.steps / (ms * 1e-3) / 1e9,
+        "unit": "GB/s", "iterations_per_s": args.steps / (ms * 1e-3), "n_gpus": world, "steps": args.steps,
+        "warmup": warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "strong",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name + "_sharded", "K": wl.K, "N": wl.N, "servers": world,
+                   "parallelism": f"{world} parameter server(s), each owning N/{world} of params and momentum; "
+                                  "gradients read through peer mappings; barrier + all-gather(params) + "
+                                  "all-reduce(norm) per step",
+                   "l2": "inputs exceed the 126 MB L2"},
+        "gpu_launches": 2 * args.steps, "clocks": sampler.summary(),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_source": f"of {peak_kind}", "kernel": "agg_vec_kernel on this rank's slice; the step "
+                     "also contains the collectives, so this is a lower bound of the kernel's own rate",
+                     "traffic": None},
+    }
+
+
 def run_ours(args):
     from paper_2305_12213_b200 import binding, build
     rank, local_rank, world = replicas.env_world()
@@ -506,7 +565,11 @@ def run_ours(args):
         build.build()
     replicas.barrier(dev)
     binding.lib()
-    if args.workload == "softmax":
+    if args.mode == "sharded":
+        out = measure_sharded(args, dev, rank, world)
+        if rank == 0:
+            print(json.dumps(out), flush=True)
+    elif args.workload == "softmax":
         out = measure_softmax(args, dev, rank, world)
         if rank == 0:
             print(json.dumps(out), flush=True)
@@ -648,6 +711,10 @@ def main():
                          "tensors (resnet50, bert_base); nonorm = the headline kernel without the gradient norm, "
                          "persistent / staged = the launch shapes measured against it and not adopted "
                          "(db_bench_aggregate_variant; fp32, no norm)")
+    ap.add_argument("--mode", choices=["replicas", "sharded"], default="replicas",
+                    help="with several GPUs: replicas = every rank runs its own independent step (default, no "
+                         "collective on the data path); sharded = one parameter server per GPU, each owning a slice "
+                         "of the model (paper_2305_12213_b200.sharded), resnet50 workload only")
     ap.add_argument("--stage-floats", type=int, choices=[512, 1024, 2048], default=512,
                     help="with --variant staged: floats per stream and CTA staged in shared memory")
     ap.add_argument("--sweep-dtype", choices=["fp32", "bf16"], default="fp32",

@@ -208,6 +208,25 @@ db_status db_aggregate_update_static(const void* const* grads,
                                      double* grad_sqnorm, void* cuda_stream);
 
 /* ------------------------------------------------------------------------
+ * Several parameter servers      (Section 4, experimental setup: the number
+ * of parameter servers is scaled so that they are not the bottleneck)
+ *
+ * The step is element-wise over the parameters, so G servers can each own a
+ * contiguous slice of params and momentum and run db_aggregate_update_ex on
+ * it, with grads[k] pointing at the same slice of worker k's buffer (on
+ * another GPU of the node: a peer mapping; the kernel reads it with ordinary
+ * loads).  db_shard_range gives the slice of server r: equal chunks of
+ * ceil(N / G) elements rounded up to a multiple of `align` (use 8: slices of
+ * 16-byte-aligned fp32 and bf16 buffers then stay on the 128-bit path), the
+ * last ones shorter or empty.  The union of the G slices is [0, N) and the
+ * results are bit-identical to one call over all N (the norm is the sum of
+ * the slices' norms).
+ *   N >= 0, G >= 1, 0 <= r < G, align >= 1, else DB_ERR_ARG; begin, end: host.
+ * ------------------------------------------------------------------------ */
+db_status db_shard_range(int64_t N, int32_t G, int32_t r, int32_t align,
+                         int64_t* begin, int64_t* end);
+
+/* ------------------------------------------------------------------------
  * The same step with the gradients in HOST memory   (Section 3.1, Eq. 2-3;
  * in the paper's system the parameter server receives the workers' gradients
  * over the network, i.e. in host buffers, and sends the new model back)

@@ -54,6 +54,15 @@ db_status db_bench_aggregate_variant(db_bench_variant variant, int32_t stage_flo
                                      float* momentum, float lr, float mu,
                                      int32_t* status, void* cuda_stream);
 
+/* The time-limited wait of the tensor-core kernels, made to run out: one CTA
+ * waits on an mbarrier that nothing ever arrives on, gives up after limit_ns
+ * nanoseconds (at most 2e9), writes `code` to *status (device int32, zeroed by
+ * the caller) and returns normally.  This is how those kernels report a wait
+ * that never ends -- a status word the host reads, the context stays usable --
+ * and the only way to see that path taken without a faulty kernel. */
+db_status db_bench_wait_timeout(int32_t* status, int32_t code, uint64_t limit_ns,
+                                void* cuda_stream);
+
 #if defined(__GNUC__)
 #pragma GCC visibility pop
 #endif

@@ -50,8 +50,10 @@ _SIGNATURES = {
     "db_multi_plan_destroy": (c_int32, [c_void_p]),
     "db_aggregate_update_static": (c_int32, [c_void_p, c_int32, c_void_p, c_int32, c_int64, c_void_p,
                                              c_void_p, c_float, c_float, c_void_p, c_void_p]),
+    "db_shard_range": (c_int32, [c_int64, c_int32, c_int32, c_int32, c_void_p, c_void_p]),
     "db_bench_read_probe_sink_bytes": (c_size_t, [c_size_t]),
     "db_bench_read_probe": (c_int32, [c_void_p, c_size_t, c_void_p, c_void_p]),
+    "db_bench_wait_timeout": (c_int32, [c_void_p, c_int32, ctypes.c_uint64, c_void_p]),
     "db_bench_aggregate_variant": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_int32, c_int64, c_void_p,
                                              c_void_p, c_float, c_float, c_void_p, c_void_p]),
     "db_host_pipeline_create": (c_int32, [c_void_p]),
@@ -206,6 +208,13 @@ def aggregate_update_static(grads: Sequence[torch.Tensor], b: Sequence[int], par
         float(lr), float(mu), _dev_ptr(grad_sqnorm, torch.float64, "grad_sqnorm"), _stream_ptr(stream)))
 
 
+def shard_range(N: int, G: int, r: int, align: int = 8):
+    """db_shard_range: the slice [begin, end) of N parameters that parameter server r of G owns."""
+    lo, hi = ctypes.c_int64(0), ctypes.c_int64(0)
+    _check(lib().db_shard_range(int(N), int(G), int(r), int(align), ctypes.byref(lo), ctypes.byref(hi)))
+    return int(lo.value), int(hi.value)
+
+
 DB_BENCH_PERSISTENT, DB_BENCH_BULK_STAGED = 1, 2
 
 
@@ -221,6 +230,13 @@ def bench_read_probe(src: torch.Tensor, sink: torch.Tensor, stream: Optional[tor
     if sink.numel() * sink.element_size() < bench_read_probe_sink_bytes(nbytes):
         raise ValueError("sink too small")
     _check(lib().db_bench_read_probe(src.data_ptr(), nbytes, sink.data_ptr(), _stream_ptr(stream)))
+
+
+def bench_wait_timeout(status: torch.Tensor, code: int, limit_ns: int,
+                       stream: Optional[torch.cuda.Stream] = None) -> None:
+    """db_bench_wait_timeout: run the kernels' bounded wait until it gives up and reports `code`."""
+    _check(lib().db_bench_wait_timeout(_dev_ptr(status, torch.int32, "status"), int(code), int(limit_ns),
+                                       _stream_ptr(stream)))
 
 
 def bench_aggregate_variant(variant: int, stage_floats: int, grads: Sequence[torch.Tensor], b: Sequence[int],

@@ -9,6 +9,7 @@
 #include "agg_device.cuh"
 #include "common.h"
 #include "dynbatch_bench.h"
+#include "tc_gemm.cuh"
 
 namespace dynbatch {
 namespace {
@@ -191,6 +192,23 @@ __global__ void __launch_bounds__(THREADS) bulk_staged_kernel(const __grid_const
     }
 }
 
+// One warp; lane 0 waits on a barrier that is never completed, with the kernels' own bounded wait.
+__global__ void __launch_bounds__(32) wait_timeout_kernel(int* status, int code, unsigned long long limit_ns) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ volatile int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        tc::mbar_init(&bar, 1);
+        tc::fence_barrier_init();
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) {
+        const bool completed = tc::mbar_wait(&bar, 0, &abort_flag, status, code, limit_ns);
+        if (completed) atomicExch(status, -1);      // cannot happen: nothing arrives
+    }
+    __syncwarp();
+}
+
 using VariantFn = void (*)(const VariantArgs);
 
 template <int K>
@@ -256,6 +274,16 @@ extern "C" db_status db_bench_read_probe(const void* src, size_t bytes, void* si
     if (ctas > 0x7fffffffLL) return DB_ERR_ARG;
     read_probe_kernel<<<static_cast<unsigned int>(ctas), kBlock, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
         static_cast<const uint4*>(src), static_cast<long long>(bytes / 16), static_cast<unsigned long long*>(sink));
+    DB_CUDA_TRY(cudaGetLastError());
+    return DB_OK;
+}
+
+extern "C" db_status db_bench_wait_timeout(int32_t* status, int32_t code, uint64_t limit_ns, void* cuda_stream) {
+    using namespace dynbatch;
+    if (!status) return DB_ERR_NULL;
+    if (code == 0 || limit_ns == 0 || limit_ns > tc::kWaitLimitNs || reinterpret_cast<uintptr_t>(status) % 4)
+        return DB_ERR_ARG;
+    wait_timeout_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(status, code, limit_ns);
     DB_CUDA_TRY(cudaGetLastError());
     return DB_OK;
 }

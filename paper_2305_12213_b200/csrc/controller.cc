@@ -121,6 +121,20 @@ extern "C" db_status db_controller_step(int32_t* b, const double* throughputs,
 }
 
 // ---------------------------------------------------------------------------
+// Slice of the parameters owned by one of several parameter servers (Section 4)
+// ---------------------------------------------------------------------------
+extern "C" db_status db_shard_range(int64_t N, int32_t G, int32_t r, int32_t align, int64_t* begin, int64_t* end) {
+    if (!begin || !end) return DB_ERR_NULL;
+    if (N < 0 || G < 1 || r < 0 || r >= G || align < 1) return DB_ERR_ARG;
+    int64_t chunk = (N + G - 1) / G;
+    chunk = (chunk + align - 1) / align * align;
+    const int64_t lo = static_cast<int64_t>(r) * chunk, hi = lo + chunk;
+    *begin = lo < N ? lo : N;
+    *end = hi < N ? hi : N;
+    return DB_OK;
+}
+
+// ---------------------------------------------------------------------------
 // Static open-loop allocation (Section 3.2)
 // ---------------------------------------------------------------------------
 extern "C" db_status db_static_allocate(const double* throughputs, int32_t K, int32_t b0,

@@ -75,9 +75,9 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-// Waits for the barrier phase; gives up after kWaitLimitNs or when another thread already did.
+// Waits for the barrier phase; gives up after limit_ns or when another thread already did.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status, int code) {
+                                          int* status, int code, unsigned long long limit_ns = kWaitLimitNs) {
     unsigned long long t0 = 0;
     for (unsigned int spin = 0;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -85,7 +85,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         if ((spin & 255u) == 255u) {
             const unsigned long long now = global_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) {
+            else if (now - t0 > limit_ns) {
                 *abort_flag = 1;
                 if (status) atomicCAS(status, 0, code);
                 return false;

@@ -61,3 +61,33 @@ def test_read_probe_reads_every_byte_it_is_given():
         assert sink.any().item(), pos
     with pytest.raises(binding.DynbatchError):
         binding.bench_read_probe(src[:100], sink)     # not a multiple of 16 bytes
+
+
+def test_a_wait_that_never_ends_gives_up_and_reports():
+    """The tensor-core kernels bound every mbarrier wait and report a time-out through a status word.
+    Here the wait is made to run out on purpose (nothing ever arrives), with a short limit: the kernel
+    returns normally, the code is in the status word, and the device goes on working."""
+    import time
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    binding.bench_wait_timeout(status, 77, 50_000_000)          # 50 ms
+    torch.cuda.synchronize()
+    waited = time.perf_counter() - t0
+    assert int(status.item()) == 77
+    assert 0.04 < waited < 1.5
+    # the first code stays: a second time-out does not overwrite it
+    binding.bench_wait_timeout(status, 78, 1_000_000)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 77
+    # the context is intact: an ordinary step runs and is right
+    N = 4096
+    g = [torch.ones(N, device=DEV) for _ in range(2)]
+    p, v = torch.zeros(N, device=DEV), torch.zeros(N, device=DEV)
+    binding.aggregate_update(g, [1, 1], p, v, 0.5, 0.0)
+    torch.cuda.synchronize()
+    assert torch.equal(v, torch.ones(N, device=DEV))
+    with pytest.raises(binding.DynbatchError):
+        binding.bench_wait_timeout(status, 0, 1000)
+    with pytest.raises(binding.DynbatchError):
+        binding.bench_wait_timeout(status, 5, 3_000_000_000)     # beyond the kernels' own 2 s limit
