@@ -91,9 +91,9 @@ WORKLOADS = {"resnet50": resnet50_workload, "bert_base": bert_base_workload, "sm
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the aggregation kernel on the
 # resnet50 workload, from the ncu capture summarised under profiles/, with the digest of the kernel
-# sources (aggregate.cu, agg_device.cuh) the counters belong to.  Reported as null once the source has changed.
-NCU_TRAFFIC = {"workload": "resnet50_arena_N25557032_K8_fp32_gbatch256", "bytes_per_launch": 1202312704,
-               "kernel_source_sha256": "896b73941fef77edddd1df2a1cbe721c689a72c93cabf6b0c7f6fd7ca0346c6b"}
+# sources (agg_kernels.cuh, agg_device.cuh) the counters belong to.  Reported as null once the source has changed.
+NCU_TRAFFIC = {"workload": "resnet50_arena_N25557032_K8_fp32_gbatch256", "bytes_per_launch": 1022323968 + 179025920,
+               "kernel_source_sha256": "368cb58fe34769104a355d122e8670135cbfd7bc17cc53e2a07046cc330e44d7"}
 
 
 NOMINAL_HBM_GBS = 8000.0   # NVIDIA's published HBM3e figure for B200 (not verifiable here): context beside the measured peak
@@ -152,7 +152,7 @@ def kernel_traffic(workload_name):
         return None
     h = hashlib.sha256()
     try:
-        for name in ("aggregate.cu", "agg_device.cuh"):
+        for name in ("agg_kernels.cuh", "agg_device.cuh"):
             with open(os.path.join(ROOT, "paper_2305_12213_b200", "csrc", name), "rb") as f:
                 h.update(f.read())
     except OSError:
