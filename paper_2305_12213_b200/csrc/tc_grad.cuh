@@ -20,8 +20,10 @@
 // accumulators; two thirds of the operand traffic of 128 x 64 tiles and 1.4 us less on the step of the
 // 256-sample check model), else 128 x 64 with up to seven accumulators.
 //
-// 192 threads: warp 0 (one lane) issues the TMA copies, warp 1 owns the tensor-memory allocation
-// and (one lane) issues the products, warps 2-5 are the epilogue.  Three shared-memory stages of
+// 320 threads: warp 0 (one lane) issues the TMA copies, warp 1 owns the tensor-memory allocation
+// and (one lane) issues the products, warps 2-9 are the epilogue (two per tensor-memory lane quarter,
+// half of the tile's columns each: 0.35 us less on the step than four warps; sending each 32-column box off as
+// soon as it is staged, instead of the whole tile at once, gained nothing).  Three shared-memory stages of
 // 16 samples; two (wide tile) or three CTAs fit on an SM and their phases (copy, products, epilogue)
 // overlap.  Measured with a time stamp per phase, a CTA is a chain of latencies rather than a stream:
 // 1 us from the predecessor's end to the first copy instruction, 1 - 2 us until the first stage has
@@ -50,7 +52,7 @@ constexpr int kStages = 3;
 constexpr int kChunkBytes = kRowsPerStage * 128;            // one [16 x 32] block of a stage
 constexpr int kAChunks = kTileM / kChunk;
 constexpr int kABytes = kAChunks * kChunkBytes;             // X_hi (or X_lo) part of a stage
-constexpr int kEpilogueWarps = 4;
+constexpr int kEpilogueWarps = 8;      // two per tensor-memory lane quarter, half of the tile's columns each
 constexpr int kEpilogueThreads = kEpilogueWarps * 32;
 constexpr int kThreads = 64 + kEpilogueThreads;
 
@@ -282,18 +284,19 @@ grad_tma_kernel(const __grid_constant__ GradArgs g) {
         }
     } else {
         // ------------------------------------------------------------ epilogue
-        const int et = tid - 64;                     // 0..127
+        const int et = tid - 64;                     // 0..255
         const int quarter = warp & 3;                // the tensor-memory lanes this warp may read
+        const int col_half = (warp - 2) >> 2;        // which half of the tile's columns it drains
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         const int row = quarter * 32 + lane;
         float* srow = reinterpret_cast<float*>(tiles) + row * kStagePitch;
-        // the verdict is made the same for all four warps (a barrier that ANDs their predicates): what
+        // the verdict is made the same for all eight warps (a barrier that ANDs their predicates): what
         // follows has warp-wide instructions and a barrier among them
         if (epilogue_all(tc::mbar_wait(&done_bar, 0, &abort_flag, g.status, 6))) {
             tc::tc_fence_after();
             const int used = min(g.n_acc, (steps * kStepRows + kAccRows - 1) / kAccRows);
 #pragma unroll 1
-            for (int c0 = 0; c0 < TILE_N; c0 += 32) {
+            for (int c0 = col_half * (TILE_N / 2); c0 < (col_half + 1) * (TILE_N / 2); c0 += 32) {
                 uint32_t r[32], x[32];
                 __syncwarp();
                 tc::tmem_load32(lane_base + g.n_acc * TILE_N + c0, r);
