@@ -260,10 +260,15 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
         kernel_label = "persistent_kernel" if variant == "persistent" else f"bulk_staged_kernel[{args.stage_floats} floats]"
     with_norm = variant in ("momentum", "adam", "tensor_list")
 
+    if variant == "momentum":
+        call = binding.AggregateStep(grads, p, v, sq, ws, stream)      # the tensors' pointers, marshalled once
+
     def step():
         nonlocal b, adam_t
         b = binding.controller_step(b, wl.throughputs, wl.kp)
-        if variant == "adam":
+        if variant == "momentum":
+            call.run(b, wl.lr, wl.mu)
+        elif variant == "adam":
             adam_t += 1
             binding.aggregate_adam(grads, b, p, v, u, 1e-3, 0.9, 0.999, 1e-8, adam_t, sq, ws, stream)
         elif variant == "tensor_list":
@@ -450,13 +455,15 @@ def measure_e2e(wl, args, dev, grads, p, v, b):
     for _ in range(2):
         e2e_step()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(dev.index)
     replicas.barrier(dev)
     torch.cuda.synchronize()
-    e0.record(stream)
-    for _ in range(e2e_steps):
-        e2e_step()
-    e1.record(stream)
-    torch.cuda.synchronize()
+    with sampler:
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        torch.cuda.synchronize()
     replicas.barrier(dev)
     e2e_ms = e0.elapsed_time(e1)
     assert np.isfinite(float(host_sq[0])) and float(host_sq[0]) > 0 and bool(torch.isfinite(host_p[:1024]).all())
@@ -466,7 +473,7 @@ def measure_e2e(wl, args, dev, grads, p, v, b):
     return {"value": e2e_bps / 1e9, "unit": "GB/s", "steps": e2e_steps, "ms_per_step": e2e_max_ms / e2e_steps,
             "h2d_bytes_per_step": K * N * wl.grad_bytes, "d2h_bytes_per_step": N * 4 + 8,
             "api": "db_aggregate_update_host, 2^21-element chunks, pinned host buffers",
-            "gpu_launches_per_step": nchunks + 1}
+            "gpu_launches_per_step": nchunks + 1, "clocks": sampler.summary()}
 
 
 def measure_softmax(args, dev, rank, world):

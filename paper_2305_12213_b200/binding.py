@@ -164,6 +164,37 @@ def aggregate_update(grads: Sequence[torch.Tensor], b: Sequence[int], params: to
         _stream_ptr(stream)))
 
 
+class AggregateStep:
+    """db_aggregate_update_ex with its tensor arguments marshalled once: for loops that call the step
+    on the same buffers every iteration (the pointers, not the tensors' contents, are fixed here).
+    `run(b, lr, mu)` then only converts the batch sizes and the two scalars."""
+
+    def __init__(self, grads: Sequence[torch.Tensor], params: torch.Tensor, momentum: torch.Tensor,
+                 grad_sqnorm: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                 stream: Optional[torch.cuda.Stream] = None):
+        self.K = len(grads)
+        gdt = grads[0].dtype
+        if gdt not in (torch.float32, torch.bfloat16):
+            raise TypeError("gradients must be float32 or bfloat16")
+        self._keep = (list(grads), params, momentum, grad_sqnorm, workspace)       # the buffers stay alive
+        self._table = (c_void_p * self.K)(*[_dev_ptr(g, gdt, "grads[k]") for g in grads])
+        self._b = (c_int32 * self.K)()
+        self._fn = lib().db_aggregate_update_ex
+        self._args = (ctypes.cast(self._table, c_void_p), DB_F32 if gdt == torch.float32 else DB_BF16,
+                      ctypes.cast(self._b, c_void_p), self.K, int(params.numel()),
+                      _dev_ptr(params, torch.float32, "params"), _dev_ptr(momentum, torch.float32, "momentum"))
+        self._tail = (_dev_ptr(grad_sqnorm, torch.float64, "grad_sqnorm"),
+                      None if workspace is None else workspace.data_ptr(),
+                      0 if workspace is None else workspace.numel() * workspace.element_size(),
+                      _stream_ptr(stream))
+
+    def run(self, b: Sequence[int], lr: float, mu: float) -> None:
+        if len(b) != self.K:
+            raise ValueError("len(b) != number of gradient buffers")
+        self._b[:] = b
+        _check(self._fn(*self._args, lr, mu, *self._tail))
+
+
 def aggregate_adam(grads: Sequence[torch.Tensor], b: Sequence[int], params: torch.Tensor,
                    first_moment: torch.Tensor, second_moment: torch.Tensor, lr: float, beta1: float,
                    beta2: float, eps: float, step: int, grad_sqnorm: Optional[torch.Tensor] = None,

@@ -214,6 +214,27 @@ def test_short_form_matches_full_form():
     assert torch.equal(p1, p2) and torch.equal(v1, v2)
 
 
+def test_prepared_step_is_the_same_call():
+    """binding.AggregateStep marshals the tensors once; every run must be the plain call's result."""
+    N, K = 300_007, 5
+    g = inputs.worker_gradients(K, N, 1e-3, 97, device=DEV, dtype=torch.bfloat16)
+    p0, v0 = inputs.normal(N, 0.02, 18, DEV), inputs.normal(N, 0.01, 19, DEV)
+    p1, v1, p2, v2 = p0.clone(), v0.clone(), p0.clone(), v0.clone()
+    sq1 = torch.zeros(1, dtype=torch.float64, device=DEV)
+    sq2 = torch.zeros(1, dtype=torch.float64, device=DEV)
+    ws1, ws2 = _workspace(K, N), _workspace(K, N)
+    step = binding.AggregateStep(g, p2, v2, sq2, ws2)
+    for b in ([3, 9, 0, 18, 5], [7, 7, 7, 7, 7]):
+        binding.aggregate_update(g, b, p1, v1, 0.1, 0.9, sq1, ws1)
+        step.run(b, 0.1, 0.9)
+        torch.cuda.synchronize()
+        assert torch.equal(p1, p2) and torch.equal(v1, v2) and float(sq1.item()) == float(sq2.item())
+    with pytest.raises(ValueError):
+        step.run([1, 2], 0.1, 0.9)
+    with pytest.raises(binding.DynbatchError):
+        step.run([0] * K, 0.1, 0.9)
+
+
 def test_on_a_side_stream():
     N, K = 500_000, 4
     g = inputs.worker_gradients(K, N, 1.0, 96, device=DEV)
