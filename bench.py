@@ -172,6 +172,7 @@ class ClockSampler:
         self.samples, self.reasons = [], set()
         self.max_mhz = None
         self._stop = threading.Event()
+        self._go = threading.Event()
         self._thread = None
         self.period = period_s
         try:
@@ -183,11 +184,20 @@ class ClockSampler:
                 index = int(visible.split(",")[index])
             self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
             self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            # the first queries of a process take milliseconds: make them here, not inside a timed region
+            pynvml.nvmlDeviceGetClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            pynvml.nvmlDeviceGetCurrentClocksEventReasons(self.h)
         except Exception:
             self.nv = None
+        if self.nv is not None:
+            # the thread exists before the region opens, so that entering the region costs the timed thread
+            # one Event.set() and not a thread start
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
 
     def _loop(self):
         nv = self.nv
+        self._go.wait()
         while not self._stop.is_set():
             try:
                 self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
@@ -200,13 +210,12 @@ class ClockSampler:
             self._stop.wait(self.period)
 
     def __enter__(self):
-        if self.nv is not None:
-            self._thread = threading.Thread(target=self._loop, daemon=True)
-            self._thread.start()
+        self._go.set()
         return self
 
     def __exit__(self, *exc):
         self._stop.set()
+        self._go.set()
         if self._thread is not None:
             self._thread.join()
 
