@@ -6,6 +6,7 @@ it imports nothing from it.  Arrays are numpy; gradients are float32 arrays or
 uint16 arrays holding bf16 bit patterns.
 """
 import ctypes
+import os
 from ctypes import POINTER, c_double, c_int32, c_int64, c_void_p
 
 import numpy as np
@@ -21,7 +22,9 @@ _lib = None
 def lib():
     global _lib
     if _lib is None:
-        L = ctypes.CDLL(_build())
+        # REF_ORACLE_LIB: a library built elsewhere from a (deliberately altered) copy of
+        # ref_oracle.c -- how tests/test_oracle_mutations.py shows that the pins catch mistakes.
+        L = ctypes.CDLL(os.environ.get("REF_ORACLE_LIB") or _build())
         L.ref_weights.argtypes = [c_void_p, c_int32, c_void_p]
         L.ref_aggregate_update.argtypes = [
             c_void_p, c_int32, c_void_p, c_int32, c_int64, c_void_p, c_void_p,

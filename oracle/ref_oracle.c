@@ -33,7 +33,11 @@
  * 3.3), sum conservation, exhaustive check of the integer apportionment;
  * for the stabilised controller pandas' EWMA, the dead-band at 0.05 and three
  * traces worked by hand (learnt bounds that cannot hold the global batch, a
- * bound learnt twice, the smoothed comparison at every observation).
+ * bound learnt twice, the smoothed comparison at every observation), the
+ * dead-band's exact form (largest relative move, against the batch in use,
+ * strictly above the threshold) and the return of surplus units.
+ * tests/test_oracle_mutations.py plants single errors in a copy of this file
+ * and requires the pins to fail for each.
  * Nothing here is left "parity unpinned".
  *
  * Build: gcc -O2 -ffp-contract=off -fopenmp -shared -fPIC (see build.py).

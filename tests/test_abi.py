@@ -195,6 +195,8 @@ def test_static_allocate_matches_oracle_and_the_papers_clusters(lib):
         b0 = int(rng.integers(1, 200))
         lo = [int(v) for v in rng.integers(0, b0 // 2 + 1, size=K)] if trial % 3 == 0 else None
         hi = [int(v) for v in rng.integers(b0, 4 * b0 + 1, size=K)] if trial % 4 == 0 else None
+        if trial % 5 == 1:                      # lower bounds above many targets: surplus units are taken back
+            lo = [int(v) for v in rng.integers(0, b0 + 1, size=K)]
         try:
             ref = oracle.static_allocate(X, b0, lo, hi).tolist()
         except oracle.OracleError as e:
@@ -205,6 +207,10 @@ def test_static_allocate_matches_oracle_and_the_papers_clusters(lib):
         assert binding.static_allocate(X, b0, lo, hi) == ref
     with pytest.raises(binding.DynbatchError):
         binding.static_allocate([1.0, -1.0], 8)
+    # surplus units after lower bounds above the targets (worked by hand in tests/test_oracle_pins.py)
+    assert binding.controller_step([4, 4, 4], [1.0, 1.0, 10.0], 1.0, [3, 1, 1], [12, 12, 12]) == [3, 1, 8]
+    assert binding.static_allocate([12.0, 13.0, 71.0], 8, [5, 1, 1], [24, 24, 24]) == [5, 2, 17]
+    assert binding.static_allocate([1.0, 1.0, 6.0], 8, [6, 1, 1], [24, 24, 24]) == [6, 1, 17]
 
 
 @pytest.mark.parametrize("seed", range(40))
@@ -276,6 +282,12 @@ HAND_TRACES = [
     ([40, 60], dict(kp=1.0, alpha=0.5, dead_band=0.35, adaptive_b_max=True),
      [[8.0, 16.0], [9.0, 10.75], [13.0, 10.75], [14.0, 10.75]],
      [[57, 43], [57, 43], [57, 43], [40, 60]]),
+    # the dead-band takes the largest relative move, a decrease included, strictly above the threshold and
+    # relative to the batch in use: (101, 9) is -10 %; (21, 19) and (19, 21) are exactly 5 %; (22, 18) is 10 %
+    ([100, 10], dict(kp=1.0, alpha=1.0, dead_band=0.05), [[100 / 101.0, 10 / 9.0]], [[101, 9]]),
+    ([20, 20], dict(kp=1.0, alpha=1.0, dead_band=0.05), [[20 / 21.0, 20 / 19.0]], [[20, 20]]),
+    ([20, 20], dict(kp=1.0, alpha=1.0, dead_band=0.05), [[20 / 19.0, 20 / 21.0]], [[20, 20]]),
+    ([20, 20], dict(kp=1.0, alpha=1.0, dead_band=0.05), [[20 / 22.0, 20 / 18.0]], [[22, 18]]),
 ]
 
 

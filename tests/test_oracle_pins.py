@@ -188,6 +188,18 @@ def test_adam_matches_torch_adam():
     assert np.allclose(p, w.detach().numpy(), rtol=1e-10, atol=1e-14)
 
 
+def test_adam_reports_the_aggregate_and_its_squared_norm():
+    """The Adam call returns the same g and sum g^2 as the momentum call: g_k = c_k everywhere gives
+    g = sum lambda_k c_k and ||g||^2 = n g^2."""
+    n, b, c = 37, [1, 3], [2.0, -6.0]                      # g = 0.25 * 2 - 0.75 * 6 = -4
+    gs = [np.full(n, v, dtype=np.float32) for v in c]
+    p, m, u = np.zeros(n), np.zeros(n), np.zeros(n)
+    g, sq = oracle.aggregate_adam(gs, b, p, m, u, 1e-3, 0.9, 0.999, 1e-8, 1, want_g=True)
+    assert np.array_equal(g, np.full(n, -4.0)) and sq == 16.0 * n
+    # first step of Adam from zero state: mhat = g, uhat = g^2, so p = -lr * g / (|g| + eps)
+    assert np.allclose(p, 1e-3 * 4.0 / (4.0 + 1e-8), rtol=1e-14)
+
+
 # ---------------------------------------------------------------- linear-softmax gradient
 def _brute_force_grad(X, y, W):
     """Per-sample definition in fp64: mean_i outer(x_i, softmax(x_i W) - onehot(y_i))."""
@@ -354,6 +366,8 @@ def test_integer_apportionment_is_optimal_exhaustively():
         X = rng.uniform(0.2, 5.0, size=K)
         kp = float(rng.choice([0.3, 0.5, 1.0]))
         lo = rng.integers(0, 2, size=K) if trial % 3 == 0 else np.ones(K, dtype=int)
+        if trial % 5 == 1:
+            lo = rng.integers(0, 4, size=K)          # lower bounds above the targets: units must be taken back
         hi = np.minimum(rng.integers(2, 9, size=K), S) if trial % 2 == 0 else np.full(K, S)
         hi = np.maximum(hi, lo)
         q = oracle.controller_targets(b, X, kp)
@@ -369,11 +383,36 @@ def test_integer_apportionment_is_optimal_exhaustively():
         assert cost <= _brute_force_best(q, S, lo, hi) + 1e-9
 
 
+def test_apportionment_takes_surplus_units_back():
+    """Lower bounds above the real targets leave too many units after the first pass; they come back from
+    the workers above their lower bound, largest excess over the target first.
+    (a) b = (4, 4, 4), X = (1, 1, 10): q = (1, 1, 10).  With b_min = (3, 1, 1) the start is (3, 1, 10) = 14;
+        workers 0 and 1 sit on their bounds, so both units come from worker 2: (3, 1, 8).
+    (b) X = (12, 13, 71), S = 24: q = X / 4 = (3, 3.25, 17.75) exactly.  With b_min = (5, 1, 1) the start is
+        (5, 3, 17) = 25.  Worker 0 has the largest excess (2) but is on its bound; of the others worker 1
+        (excess -0.25) gives the unit, not worker 2 (-0.75): (5, 2, 17), the nearest feasible vector.
+    (c) q = (3, 3, 18), b_min = (6, 1, 1): start (6, 3, 18) = 27; equal excesses go lowest index first:
+        worker 1, then worker 2 (0 against -1), then worker 1 again: (6, 1, 17)."""
+    q = oracle.controller_targets([4, 4, 4], [1.0, 1.0, 10.0], 1.0)
+    assert np.abs(q - [1.0, 1.0, 10.0]).max() < 1e-12
+    assert oracle.controller_step([4, 4, 4], [1.0, 1.0, 10.0], 1.0, [3, 1, 1], [12, 12, 12]).tolist() == [3, 1, 8]
+    assert oracle.static_allocate([12.0, 13.0, 71.0], 8, [5, 1, 1], [24, 24, 24]).tolist() == [5, 2, 17]
+    assert oracle.static_allocate([1.0, 1.0, 6.0], 8, [6, 1, 1], [24, 24, 24]).tolist() == [6, 1, 17]
+
+
 def test_apportionment_ties_go_to_lowest_index():
     # q = (2.5, 2.5, 7.5, 7.5): two spare units, four equal remainders
     assert oracle.static_allocate([1, 1, 3, 3], 5).tolist() == [3, 3, 7, 7]
     # q = (2.5, 2.5, 2.5, 2.5) from b = (2, 2, 3, 3) with equal throughputs
     assert oracle.controller_step([2, 2, 3, 3], [1.0, 1.0, 1.0, 1.0], 1.0).tolist() == [3, 3, 2, 2]
+
+
+def test_without_bounds_every_worker_keeps_at_least_one_sample():
+    """A worker 1000 times slower has a real target of 16/1001 < 0.5; with no bounds given it still
+    holds one sample (a worker with b = 0 would drop out of the job), and b_min = 0 allows the zero."""
+    assert oracle.controller_step([8, 8], [1000.0, 1.0], 1.0).tolist() == [15, 1]
+    assert oracle.controller_step([8, 8], [1000.0, 1.0], 1.0, [0, 0], [16, 16]).tolist() == [16, 0]
+    assert oracle.static_allocate([1000.0, 1.0], 8).tolist() == [15, 1]
 
 
 def test_controller_rejects_bad_arguments():
@@ -430,6 +469,24 @@ def test_dead_band_holds_small_changes_and_passes_large_ones():
     assert st.observe([1.00, 1.03]) is False and st.b.tolist() == [100, 100]
     assert st.observe([1.0, 2.0]) is True
     assert st.b.tolist() == [133, 67] and int(st.n_since[0]) == 0
+
+
+def test_dead_band_measures_the_largest_relative_move_against_the_current_batch():
+    """Section 3.3.1, step 4: max_k |b'_k - b_k| / b_k > dmin, strictly, relative to the batch in use.
+    (a) The largest relative move may be a decrease: b = (100, 10) -> (101, 9) is +1 % and -10 %.
+    (b) b = (20, 20) -> (21, 19) moves both workers by exactly 1/20 = 0.05: not above 0.05, nothing
+        changes (measured against the new batch 1/19 > 0.05 would readjust).
+    (c) b = (20, 20) -> (19, 21) likewise; one more unit, (22, 18), is 10 % and readjusts."""
+    # (a) times chosen so that the targets are q = (101, 9): X proportional to (101, 9)
+    st = oracle.ControllerState([100, 10], kp=1.0, alpha=1.0, dmin=0.05)
+    assert st.observe([100 / 101.0, 10 / 9.0]) is True and st.b.tolist() == [101, 9]
+    # (b), (c)
+    for X, moved in (((21.0, 19.0), [21, 19]), ((19.0, 21.0), [19, 21])):
+        assert oracle.controller_step([20, 20], X, 1.0).tolist() == moved
+        st = oracle.ControllerState([20, 20], kp=1.0, alpha=1.0, dmin=0.05)
+        assert st.observe([20 / X[0], 20 / X[1]]) is False and st.b.tolist() == [20, 20]
+    st = oracle.ControllerState([20, 20], kp=1.0, alpha=1.0, dmin=0.05)
+    assert st.observe([20 / 22.0, 20 / 18.0]) is True and st.b.tolist() == [22, 18]
 
 
 def test_dead_band_stops_oscillation_under_noise():
