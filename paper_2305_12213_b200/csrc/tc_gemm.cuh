@@ -353,9 +353,12 @@ __device__ __forceinline__ void tf32x3_gemm_body(const GemmArgs& g, const int sp
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
-    // everything above overlaps the previous kernel; its outputs are read only from here on
-    griddep_launch_dependents();
+    // Everything above overlaps the previous kernel; its outputs are read only from here on.  The
+    // successor is released after the wait: as the logits kernel of a worker-gradient call it is followed
+    // by a kernel that writes the workspace before waiting, which must not start while an earlier call's
+    // kernels still read it.
     griddep_wait();
+    griddep_launch_dependents();
     // a time-out needs seconds, this store comes microseconds after the launch: no wait can have given up yet
     if (g.clear_status && tid == 0 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) *g.status = 0;
 

@@ -290,7 +290,7 @@ grad_tma_kernel(const __grid_constant__ GradArgs g) {
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         const int row = quarter * 32 + lane;
         float* srow = reinterpret_cast<float*>(tiles) + row * kStagePitch;
-        // the verdict is made the same for all eight warps (a barrier that ANDs their predicates): what
+        // the decision is made the same for all eight warps (a barrier that ANDs their predicates): what
         // follows has warp-wide instructions and a barrier among them
         if (epilogue_all(tc::mbar_wait(&done_bar, 0, &abort_flag, g.status, 6))) {
             tc::tc_fence_after();

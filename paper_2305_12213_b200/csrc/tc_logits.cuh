@@ -135,8 +135,11 @@ logits_tma_kernel(const __grid_constant__ LogitArgs g) {
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
-    tc::griddep_launch_dependents();
+    // The successor (the softmax kernel) splits X into the workspace before its own wait.  It may be
+    // scheduled only once every kernel before this one has finished -- an earlier call's gradient kernel
+    // may still be reading those arrays -- so the trigger comes after the wait, not before it.
     tc::griddep_wait();
+    tc::griddep_launch_dependents();
     // a time-out needs seconds, this store comes microseconds after the launch: no wait can have given up yet
     if (g.clear_status && tid == 0 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) *g.status = 0;
 
@@ -218,7 +221,7 @@ logits_tma_kernel(const __grid_constant__ LogitArgs g) {
         bool alive = true;
         for (int kb = 0; kb < nkb; ++kb) {
             const int s = kb % kStages;
-            // the verdict is made the same for the whole warp: what follows has warp-wide operations
+            // the decision is made the same for the whole warp: what follows has warp-wide operations
             alive = __all_sync(0xffffffffu, tc::mbar_wait(&full_bar[s], (kb / kStages) & 1, &abort_flag, g.status, 8));
             if (!alive) break;
             unsigned char* st = ring + s * L::kStage;

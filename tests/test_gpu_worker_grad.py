@@ -190,6 +190,30 @@ def test_grouped_then_aggregate_is_the_concatenated_batch_gradient():
     assert rel_err(f64(v), full.reshape(-1)) <= FP32_TOL
 
 
+def test_back_to_back_calls_on_one_workspace_do_not_disturb_each_other():
+    """Calls that share a workspace, enqueued without synchronising and with different samples: each call's
+    kernels may be scheduled under the previous call's, but none may touch the workspace before those have
+    finished.  Every call's gradients equal (bitwise) the ones it gives when run alone."""
+    bs = [24, 40, 64, 128]
+    D, C = 2048, 1000
+    offs = [0] + list(np.cumsum(bs))
+    problems = [inputs.softmax_problem(bs, D, C, seed=7000 + i, w_std=0.02, device=DEV) for i in range(3)]
+    alone = [_grouped(X, y, W, bs)[0] for X, y, W in problems]
+    ws = torch.empty(binding.worker_grad_grouped_workspace_bytes(offs[-1], len(bs), D, C), dtype=torch.uint8,
+                     device=DEV)
+    for rep in range(10):
+        outs = [[torch.full((D, C), float("nan"), device=DEV) for _ in bs] for _ in problems]
+        losses = [torch.zeros(len(bs), device=DEV) for _ in problems]
+        torch.cuda.synchronize()
+        for (X, y, W), G, l in zip(problems, outs, losses):
+            binding.worker_grad_grouped(X, y, W, offs, G, l, ws)
+        torch.cuda.synchronize()
+        assert binding.worker_grad_status(ws) == 0
+        for i, (G, ref) in enumerate(zip(outs, alone)):
+            for w in range(len(bs)):
+                assert torch.equal(G[w], ref[w]), f"repetition {rep}, call {i}, worker {w}"
+
+
 def test_grouped_argument_errors():
     X, y, W = inputs.softmax_problem([4, 4], 16, 8, seed=9, device=DEV)
     G = [torch.empty(16, 8, device=DEV) for _ in range(2)]
