@@ -75,7 +75,8 @@ typedef enum {
  *                  b[k] == 0 has weight 0 and its buffer is never read.
  *   b              host, K mini-batch sizes, each >= 0, sum > 0
  *   K              1..DB_MAX_K
- *   N              number of parameters, >= 0 (0: DB_OK, nothing enqueued)
+ *   N              number of parameters, >= 0 (0: DB_OK, nothing enqueued,
+ *                  *grad_sqnorm left as it was)
  *   params         device, N fp32, updated in place
  *   momentum       device, N fp32, updated in place
  *   lr, mu         finite learning rate and momentum coefficient
