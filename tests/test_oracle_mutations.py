@@ -2,12 +2,12 @@
 
 Each case below plants ONE plausible error in a copy of oracle/ref_oracle.c -- a dropped term, a wrong sign,
 a transposed operand, a missing normalisation -- builds the copy with the oracle's own compiler flags, and runs
-tests/test_oracle_pins.py against it in a child process (the oracle front end loads the library named by
-REF_ORACLE_LIB instead of building its own).  The pins must FAIL for every planted error and pass for an
+tests/test_oracle_pins.py against it in a child process (tests/oracle_mutation_runner.py; the oracle front end
+loads the library named by REF_ORACLE_LIB instead of building its own).  The pins must FAIL for every planted error and pass for an
 unaltered copy.  The errors live in the CPU oracle only; nothing here touches the CUDA library.
 """
+import json
 import os
-import re
 import subprocess
 import sys
 from concurrent.futures import ThreadPoolExecutor
@@ -100,43 +100,47 @@ def _mutate(text, old, new, which):
     return text[:pos] + new + text[pos + len(old):]
 
 
-def _run_pins(lib_path):
-    env = dict(os.environ, REF_ORACLE_LIB=lib_path, OMP_NUM_THREADS="1")
-    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(ROOT, "tests", "test_oracle_pins.py"), "-x", "-q",
-                        "-p", "no:cacheprovider", "--no-header"], cwd=ROOT, env=env, capture_output=True, text=True,
-                       timeout=600)
-    first = re.search(r"^FAILED (\S+)", r.stdout, re.M)
-    return r.returncode, (first.group(1).split("::")[-1] if first else ""), r.stdout[-1500:]
-
-
-def _build_and_run(args):
+def _build(args):
     name, old, new, which, workdir, source = args
     c = os.path.join(workdir, name + ".c")
     so = os.path.join(workdir, name + ".so")
     with open(c, "w") as f:
         f.write(source if old is None else _mutate(source, old, new, which))
     subprocess.run(["gcc", *CFLAGS, "-o", so, c, "-lm"], check=True)
-    return (name,) + _run_pins(so)
+    return name, so
+
+
+def _run_group(pairs):
+    """One child process runs the pin file against each library of the group in turn."""
+    env = dict(os.environ, OMP_NUM_THREADS="1")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "tests", "oracle_mutation_runner.py"),
+                        *[f"{n}={so}" for n, so in pairs]], cwd=ROOT, env=env, capture_output=True, text=True,
+                       timeout=1200)
+    rows = [json.loads(line) for line in r.stdout.splitlines() if line.startswith("{")]
+    assert r.returncode == 0 and len(rows) == len(pairs), (r.returncode, r.stdout[-1500:], r.stderr[-1500:])
+    return rows
 
 
 def test_every_planted_mistake_fails_a_pin(tmp_path):
     source = open(SRC).read()
     jobs = [("unaltered", None, None, None, str(tmp_path), source)]
     jobs += [(n, o, w, i, str(tmp_path), source) for n, o, w, i in MUTATIONS]
-    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
-        results = list(pool.map(_build_and_run, jobs))
-    name, rc, _, tail = results[0]
-    assert rc == 0, "the pins do not pass on an unaltered copy of the oracle:\n" + tail
+    workers = min(4, os.cpu_count() or 1)
+    with ThreadPoolExecutor(max_workers=workers) as pool:
+        built = list(pool.map(_build, jobs))
+        groups = [built[g::workers] for g in range(workers)]
+        rows = [row for rows in pool.map(_run_group, groups) for row in rows]
+    by_name = {row["name"]: row for row in rows}
+    assert by_name["unaltered"]["rc"] == 0, "the pins do not pass on an unaltered copy of the oracle"
     # pytest exits 1 when tests ran and some failed; anything else (collection error, crash) is not a catch
-    survived = [n for n, rc, _, _ in results[1:] if rc == 0]
-    broken = [(n, rc, tail) for n, rc, _, tail in results[1:] if rc not in (0, 1)]
+    survived = [n for n, _, _, _ in MUTATIONS if by_name[n]["rc"] == 0]
+    broken = [by_name[n] for n, _, _, _ in MUTATIONS if by_name[n]["rc"] not in (0, 1)]
     assert not broken, broken
     assert not survived, f"no pin notices: {survived}"
-    caught_by = {n: first for n, _, first, _ in results[1:]}
-    assert all(caught_by.values()), caught_by
+    assert all(by_name[n]["first"] for n, _, _, _ in MUTATIONS), by_name
     with open(os.path.join(str(tmp_path), "caught_by.txt"), "w") as f:
-        for n, first in caught_by.items():
-            f.write(f"{n}\t{first}\n")
+        for n, _, _, _ in MUTATIONS:
+            f.write(f"{n}\t{by_name[n]['first']}\n")
 
 
 def test_mutations_are_distinct_and_apply():
