@@ -214,6 +214,45 @@ def test_back_to_back_calls_on_one_workspace_do_not_disturb_each_other():
                 assert torch.equal(G[w], ref[w]), f"repetition {rep}, call {i}, worker {w}"
 
 
+def test_grouped_call_and_aggregation_replay_from_a_cuda_graph():
+    """The three launches of the grouped call (tensor maps travel in the kernel parameters) and the aggregation
+    behind it can be captured once and replayed: same bits as the eager calls, replay after replay."""
+    bs = [24, 40, 64, 128]
+    D, C = 2048, 1000
+    offs = [0] + list(np.cumsum(bs))
+    X, y, W = inputs.softmax_problem(bs, D, C, seed=7100, w_std=0.02, device=DEV)
+    eager, eager_losses, _ = _grouped(X, y, W, bs)
+    N = D * C
+    ep, ev = torch.zeros(N, device=DEV), torch.zeros(N, device=DEV)
+    binding.aggregate_update([g.reshape(-1) for g in eager], bs, ep, ev, 0.5, 0.9)
+    torch.cuda.synchronize()
+
+    G = [torch.full((D, C), float("nan"), device=DEV) for _ in bs]
+    losses = torch.zeros(len(bs), device=DEV)
+    ws = torch.empty(binding.worker_grad_grouped_workspace_bytes(offs[-1], len(bs), D, C), dtype=torch.uint8,
+                     device=DEV)
+    p, v = torch.zeros(N, device=DEV), torch.zeros(N, device=DEV)
+    binding.worker_grad_grouped(X, y, W, offs, G, losses, ws)          # not the first call in capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        stream = torch.cuda.current_stream()
+        binding.worker_grad_grouped(X, y, W, offs, G, losses, ws, stream)
+        binding.aggregate_update([g.reshape(-1) for g in G], bs, p, v, 0.5, 0.9, None, None, stream)
+    for rep in range(3):
+        for g in G:
+            g.fill_(float("nan"))
+        p.zero_()
+        v.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert binding.worker_grad_status(ws) == 0
+        for w in range(len(bs)):
+            assert torch.equal(G[w], eager[w]), f"replay {rep}, worker {w}"
+        assert np.array_equal(losses.cpu().numpy(), eager_losses)
+        assert torch.equal(p, ep) and torch.equal(v, ev)
+
+
 def test_grouped_argument_errors():
     X, y, W = inputs.softmax_problem([4, 4], 16, 8, seed=9, device=DEV)
     G = [torch.empty(16, 8, device=DEV) for _ in range(2)]
