@@ -69,6 +69,8 @@ __device__ __forceinline__ double block_sum(double x, double* smem) {
 // completed and its writes are visible.
 __device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Ask the L2 to fetch the line that holds `p`; nothing is read into the SM.
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 // Gradient norm, step 1: every CTA of an aggregation kernel leaves the sum of its squared
 // aggregated gradients in partials[blockIdx.x].

@@ -30,6 +30,7 @@ struct AggArgs {
     float lr, mu;             // mu: momentum coefficient, or Adam's beta1
     float beta2, eps, inv_c1, inv_c2;   // Adam: 1 / (1 - beta^t) bias corrections
     int K;
+    int prefetch_ctas;        // CTAs [0, prefetch_ctas) ask the L2 for their state vectors before they wait
 };
 
 enum Optimizer { kMomentum = 0, kAdam = 1 };
@@ -104,9 +105,28 @@ agg_vec_kernel(const __grid_constant__ AggArgs a) {
     // the next step) may be scheduled already, and this one, if it was itself scheduled early, touches
     // memory only once its predecessor has completed.  Both are no-ops for ordinary launches.
     agg::griddep_launch_dependents();
+    const long long tile = static_cast<long long>(BLOCK) * UNROLL;
+    // On a small grid the CTAs are resident while the predecessor still runs.  They use that time to ask the
+    // L2 for their part of the state vectors (a prefetch consumes no data, so it needs no ordering against
+    // whoever may still be writing them); their loads after the wait then meet the L2 instead of DRAM.  The
+    // host sets prefetch_ctas to the grid size for such launches and to zero for all others.  (Not in the
+    // chunked kernel, KT == 0: with this block compiled in, it ran 27 % slower at N = 2^20, K = 32.)
+    if (KT > 0 && static_cast<int>(blockIdx.x) < a.prefetch_ctas) {
+#pragma unroll 1
+        for (int t = 0; t < TILES; ++t) {
+            const long long base = (static_cast<long long>(blockIdx.x) * TILES + t) * tile;
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const long long v0 = base + u * BLOCK + threadIdx.x;
+                if (v0 >= a.nvec) continue;
+                agg::prefetch_l2(reinterpret_cast<const float4*>(a.p + a.head) + v0 * kQuads);
+                agg::prefetch_l2(reinterpret_cast<const float4*>(a.v + a.head) + v0 * kQuads);
+                if (OPT == kAdam) agg::prefetch_l2(reinterpret_cast<const float4*>(a.u + a.head) + v0 * kQuads);
+            }
+        }
+    }
     agg::griddep_wait();
 
-    const long long tile = static_cast<long long>(BLOCK) * UNROLL;
 #pragma unroll 1
     for (int t = 0; t < TILES; ++t) {
         const long long base = (static_cast<long long>(blockIdx.x) * TILES + t) * tile;

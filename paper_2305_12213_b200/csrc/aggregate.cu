@@ -192,6 +192,15 @@ db_status aggregate_launch(AggArgs a, int opt, const void* const* grads, db_dtyp
         const long long tiles = (a.nvec + vectors_per_cta - 1) / vectors_per_cta;
         if (tiles > 0x7fffffffLL) return DB_ERR_ARG;
         grid = static_cast<int>(tiles < 1 ? 1 : tiles);
+        // Grids of at most one wave (what an SM's 2048 threads hold of this CTA size, on every SM) of a launch
+        // that may be scheduled under its predecessor: every CTA asks the L2 for its state vectors before it
+        // waits.  Measured on B200, steps back to back: 7.7 -> 6.8 us for N = 2^20, K = 3; 49.9 -> 44.0 us for
+        // N = 2^22, K = 16; 44.7 -> 42.5 us for the 2,048,000-parameter step behind the worker-gradient kernels.
+        // Larger grids lose: at 1.7 waves (N = 2^22, K = 2) 18.4 -> 19.1 us, and on the large workloads even the
+        // first wave alone doing so costs 3 % (ResNet-50 shapes 173.1 -> 178.8 us, BERT-base 738 -> 772 us): its
+        // CTAs then start their gradient loads in lock step.
+        const int first_wave = sm_count() * (2048 / block);
+        if (!chunk_partials && !chunk_ctas && active <= 16 && grid <= first_wave) a.prefetch_ctas = grid;
     } else {
         grid = scalar_grid(fn, N);
     }
