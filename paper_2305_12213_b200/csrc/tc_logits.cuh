@@ -17,10 +17,11 @@
 // 320 threads: warps 0-7 derive the lo halves and later drain the accumulators, warp 8 owns tensor
 // memory and (one lane) issues the products, warp 9 issues the copies: five lanes, one box each, in
 // the same instruction (measured: a further box costs about half as much that way as from the same
-// thread, and an iteration of the copy loop costs 0.3 us before its first box).  While the
-// first stage is on its way, the threads of warps 0-7 ask the L2 to prefetch every later box of the
-// CTA's share of W, one box each, so that the ring of three stages meets L2 latencies, not DRAM's
-// (issued in a row by the copying warp these requests delayed its first copy by 1.6 us).
+// thread, and an iteration of the copy loop costs 0.3 us before its first box).  Before the CTA
+// waits for its predecessor, its threads ask the L2 to prefetch every box of its share of W and X, one
+// box each, so that the ring of three stages meets L2 latencies, not DRAM's (issued in a row by the
+// copying warp these requests delayed its first copy by 1.6 us; issued after the wait instead of
+// before it the step behind a running predecessor took 0.85 us longer).
 // Every wait is bounded as in tc_gemm.cuh.
 #pragma once
 #include <cuda.h>
@@ -138,6 +139,14 @@ logits_tma_kernel(const __grid_constant__ LogitArgs g) {
     // The successor (the softmax kernel) splits X into the workspace before its own wait.  It may be
     // scheduled only once every kernel before this one has finished -- an earlier call's gradient kernel
     // may still be reading those arrays -- so the trigger comes after the wait, not before it.
+    // Before the wait, while the predecessor may still run: ask the L2 for every box of W and X this CTA will
+    // copy, one box per thread (a TMA instruction costs its thread 0.2 - 0.4 us, measured, so they are issued side
+    // by side rather than in a row by the copying warp).  A prefetch consumes no data and needs no ordering
+    // against whoever may still be writing W; the three-stage ring then meets L2 latency instead of DRAM's.
+    if (tid < nkb * kAChunks)
+        tma_prefetch_2d(&g.w, m0 + (tid % kAChunks) * 32, k_begin + (tid / kAChunks) * kBlockK);
+    else if (tid < nkb * kAChunks + nkb && tid < kSplitThreads)
+        tma_prefetch_2d(&g.x, k_begin + (tid - nkb * kAChunks) * kBlockK, n0);
     tc::griddep_wait();
     tc::griddep_launch_dependents();
     // a time-out needs seconds, this store comes microseconds after the launch: no wait can have given up yet
@@ -213,11 +222,6 @@ logits_tma_kernel(const __grid_constant__ LogitArgs g) {
         }
     } else {
         // ------------------------------------------------------------ lo halves, then the epilogue
-        // First, while the first stage is on its way: ask the L2 to fetch the boxes of W that the later
-        // stages will copy, one box per thread (a TMA instruction costs its thread 0.2 - 0.4 us, measured, so
-        // they are issued side by side here rather than in a row by the copying warp).
-        if (tid >= kAChunks && tid < nkb * kAChunks)
-            tma_prefetch_2d(&g.w, m0 + (tid % kAChunks) * 32, k_begin + (tid / kAChunks) * kBlockK);
         bool alive = true;
         for (int kb = 0; kb < nkb; ++kb) {
             const int s = kb % kStages;
