@@ -33,6 +33,10 @@ namespace {
 constexpr int kTile = 64;      // output tile edge
 constexpr int kDepth = 16;     // reduction slice per shared-memory stage
 constexpr int kThreads = 256;  // 16 x 16 threads, 4 x 4 outputs each
+// CTA of the softmax kernel (one per sample).  Measured on the 1000-class check model, step back to back:
+// 256 threads 41.7 us, 512 threads 41.0, 768 threads 42.4, 1024 threads 45.3; 128 threads (logits parked in
+// memory between the passes) 44.0.
+constexpr int kSoftmaxThreads = 512;
 
 // out[m, n] = sum_{k in split} A(m, k) * B[k, n]
 //   A(m, k) = TRANS_A ? A[k * lda + m] : A[m * lda + k];   B row-major, ldb
@@ -157,14 +161,14 @@ __device__ __forceinline__ float block_reduce(float x, float* smem, bool take_ma
     if ((threadIdx.x & 31) == 0) smem[threadIdx.x >> 5] = x;
     __syncthreads();
     float r = smem[0];
-    for (int w = 1; w < kThreads / 32; ++w) r = take_max ? fmaxf(r, smem[w]) : r + smem[w];
+    for (int w = 1; w < kSoftmaxThreads / 32; ++w) r = take_max ? fmaxf(r, smem[w]) : r + smem[w];
     return r;  // same value in every thread
 }
 
 // One CTA per sample i:  E[i, :] = (softmax(z_i) - onehot(y_i)) / b,  z_i = sum of the split partials
 // (split order).  The last CTA to finish also folds the per-sample losses into the mean loss; arrival
 // order comes from an atomic ticket (zeroed by the caller), nobody waits.
-// IN_REGS: C <= 4 * kThreads, every thread keeps its four logits in registers (one pass over memory);
+// IN_REGS: C <= 4 * kSoftmaxThreads, every thread keeps its up to four logits in registers (one pass over memory);
 // otherwise the logits are parked in E between the passes.
 // Rows [off[w], off[w + 1]) belong to worker w; each worker has its own 1/b, ticket and loss slot.
 struct RowGroups {
@@ -190,12 +194,12 @@ struct SplitOut {
 };
 
 template <bool IN_REGS, bool SPLIT>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kSoftmaxThreads)
 softmax_residual_kernel(const float* __restrict__ partials, int splits, long long split_stride,
                         const int32_t* __restrict__ y, float* __restrict__ E, float* __restrict__ row_loss,
                         const __grid_constant__ RowGroups groups, int C, unsigned int* __restrict__ tickets,
                         float* __restrict__ losses, const __grid_constant__ SplitOut so) {
-    __shared__ float smem[kThreads / 32];
+    __shared__ float smem[kSoftmaxThreads / 32];
     __shared__ float z_label;
     __shared__ bool is_last;
     tc::griddep_launch_dependents();
@@ -211,19 +215,19 @@ softmax_residual_kernel(const float* __restrict__ partials, int splits, long lon
         float* xh = so.x_hi + static_cast<long long>(ip) * so.x_pitch;
         float* xl = so.x_lo + static_cast<long long>(ip) * so.x_pitch;
         // the columns between C (D) and the pitch are copied with the rest of their 32-column chunk: zeros
-        for (int c = C + threadIdx.x; c < so.e_pitch; c += kThreads) { eh[c] = 0.0f; el[c] = 0.0f; }
-        for (int d = so.D + threadIdx.x; d < so.x_pitch; d += kThreads) { xh[d] = 0.0f; xl[d] = 0.0f; }
+        for (int c = C + threadIdx.x; c < so.e_pitch; c += kSoftmaxThreads) { eh[c] = 0.0f; el[c] = 0.0f; }
+        for (int d = so.D + threadIdx.x; d < so.x_pitch; d += kSoftmaxThreads) { xh[d] = 0.0f; xl[d] = 0.0f; }
         if (r >= groups.off[w + 1] - groups.off[w]) {
             // padding row: zeros in all four arrays (the workspace may hold anything, NaN included)
-            for (int c = threadIdx.x; c < C; c += kThreads) { eh[c] = 0.0f; el[c] = 0.0f; }
-            for (int d = threadIdx.x; d < so.D; d += kThreads) { xh[d] = 0.0f; xl[d] = 0.0f; }
+            for (int c = threadIdx.x; c < C; c += kSoftmaxThreads) { eh[c] = 0.0f; el[c] = 0.0f; }
+            for (int d = threadIdx.x; d < so.D; d += kSoftmaxThreads) { xh[d] = 0.0f; xl[d] = 0.0f; }
             return;
         }
         i = groups.off[w] + r;
         // the feature row is an input of the whole call, not of the logits kernel: split it while that runs
         const float* xr = so.X + static_cast<long long>(i) * so.D;
         if (so.x_vec) {
-            for (int d = threadIdx.x * 4; d < so.D; d += 4 * kThreads) {
+            for (int d = threadIdx.x * 4; d < so.D; d += 4 * kSoftmaxThreads) {
                 const float4 v = __ldg(reinterpret_cast<const float4*>(xr + d));
                 float4 h, l;
                 tc::split_tf32(v.x, h.x, l.x);
@@ -234,7 +238,7 @@ softmax_residual_kernel(const float* __restrict__ partials, int splits, long lon
                 *reinterpret_cast<float4*>(xl + d) = l;
             }
         } else {
-            for (int d = threadIdx.x; d < so.D; d += kThreads) tc::split_tf32(__ldg(xr + d), xh[d], xl[d]);
+            for (int d = threadIdx.x; d < so.D; d += kSoftmaxThreads) tc::split_tf32(__ldg(xr + d), xh[d], xl[d]);
         }
     } else {
         while (w + 1 < groups.K && i >= groups.off[w + 1]) ++w;
@@ -251,14 +255,14 @@ softmax_residual_kernel(const float* __restrict__ partials, int splits, long lon
     if (threadIdx.x == 0) z_label = 0.0f;
     tc::griddep_wait();      // the logits kernel has finished and its partial sums are visible
     // four classes per thread and eight splits per round: 32 independent loads in flight, adds in split order
-    for (int cb = 0; cb < C; cb += 4 * kThreads) {
+    for (int cb = 0; cb < C; cb += 4 * kSoftmaxThreads) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) z[j] = 0.0f;
         for (int s0 = 0; s0 < splits; s0 += 8) {
             float t[4][8];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const int c = cb + j * kThreads + threadIdx.x;
+                const int c = cb + j * kSoftmaxThreads + threadIdx.x;
 #pragma unroll
                 for (int u = 0; u < 8; ++u)
                     t[j][u] = (c < C && s0 + u < splits)
@@ -272,7 +276,7 @@ softmax_residual_kernel(const float* __restrict__ partials, int splits, long lon
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int c = cb + j * kThreads + threadIdx.x;
+            const int c = cb + j * kSoftmaxThreads + threadIdx.x;
             if (c < C) {
                 if (!IN_REGS) e[c] = z[j];
                 zmax = fmaxf(zmax, z[j]);
@@ -284,7 +288,7 @@ softmax_residual_kernel(const float* __restrict__ partials, int splits, long lon
     if (IN_REGS) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int c = j * kThreads + threadIdx.x;
+            const int c = j * kSoftmaxThreads + threadIdx.x;
             if (c < C) {
                 z[j] = expf(z[j] - zmax);       // numerator of the softmax
                 den += z[j];
@@ -292,7 +296,7 @@ softmax_residual_kernel(const float* __restrict__ partials, int splits, long lon
             }
         }
     } else {
-        for (int c = threadIdx.x; c < C; c += kThreads) {
+        for (int c = threadIdx.x; c < C; c += kSoftmaxThreads) {
             const float p = expf(e[c] - zmax);
             den += p;
             if (c == label) z_label = p;
@@ -304,7 +308,7 @@ softmax_residual_kernel(const float* __restrict__ partials, int splits, long lon
     if (IN_REGS) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int c = j * kThreads + threadIdx.x;
+            const int c = j * kSoftmaxThreads + threadIdx.x;
             if (c < C) {
                 float r = z[j] / den;
                 if (c == label) r -= 1.0f;
@@ -314,7 +318,7 @@ softmax_residual_kernel(const float* __restrict__ partials, int splits, long lon
             }
         }
     } else {
-        for (int c = threadIdx.x; c < C; c += kThreads) {
+        for (int c = threadIdx.x; c < C; c += kSoftmaxThreads) {
             float r = expf(e[c] - zmax) / den;
             if (c == label) r -= 1.0f;
             r *= inv_b;
@@ -331,7 +335,7 @@ softmax_residual_kernel(const float* __restrict__ partials, int splits, long lon
     if (!is_last) return;
     __threadfence();
     float part = 0.0f;
-    for (int r = threadIdx.x; r < b; r += kThreads) part += __ldcg(row_loss + row0 + r);
+    for (int r = threadIdx.x; r < b; r += kSoftmaxThreads) part += __ldcg(row_loss + row0 + r);
     const float total = block_reduce(part, smem, false);
     if (threadIdx.x == 0) *loss = total * inv_b;
 }
@@ -357,8 +361,8 @@ struct OverlappedLaunch {
 db_status launch_softmax(const float* partials, int splits, long long split_stride, const int32_t* y, float* E,
                          float* row_loss, const RowGroups& groups, int rows, int C, unsigned int* tickets,
                          float* losses, cudaStream_t stream, bool overlap, const SplitOut* split = nullptr) {
-    const bool in_regs = C <= 4 * kThreads;
-    OverlappedLaunch L(dim3(split ? groups.poff[groups.K] : rows), dim3(kThreads), 0, stream, overlap);
+    const bool in_regs = C <= 4 * kSoftmaxThreads;
+    OverlappedLaunch L(dim3(split ? groups.poff[groups.K] : rows), dim3(kSoftmaxThreads), 0, stream, overlap);
     const SplitOut so = split ? *split : SplitOut{};
     auto fn = split ? (in_regs ? softmax_residual_kernel<true, true> : softmax_residual_kernel<false, true>)
                     : (in_regs ? softmax_residual_kernel<true, false> : softmax_residual_kernel<false, false>);
