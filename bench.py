@@ -92,8 +92,8 @@ WORKLOADS = {"resnet50": resnet50_workload, "bert_base": bert_base_workload, "sm
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the aggregation kernel on the
 # resnet50 workload, from the ncu capture summarised under profiles/, with the digest of the kernel
 # sources (agg_kernels.cuh, agg_device.cuh) the counters belong to.  Reported as null once the source has changed.
-NCU_TRAFFIC = {"workload": "resnet50_arena_N25557032_K8_fp32_gbatch256", "bytes_per_launch": 1022296064 + 180271104,
-               "kernel_source_sha256": "fea992731ab401539bc690985426e04d4c70a90b9a221447423831f31b085464"}
+NCU_TRAFFIC = {"workload": "resnet50_arena_N25557032_K8_fp32_gbatch256", "bytes_per_launch": 1022299392 + 179061504,
+               "kernel_source_sha256": "102a1c7047db046edaeae11a7d165cc5883ca2431a7d4e2e43615bfd83c20af8"}
 
 
 NOMINAL_HBM_GBS = 8000.0   # NVIDIA's published HBM3e figure for B200 (not verifiable here): context beside the measured peak

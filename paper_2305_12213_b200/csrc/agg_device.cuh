@@ -101,7 +101,7 @@ static inline cudaError_t launch_norm_finalize(const double* partials, long long
     cudaLaunchConfig_t cfg{};
     cudaLaunchAttribute attr[1]{};
     cfg.gridDim = dim3(1);
-    cfg.blockDim = dim3(n > 8192 ? 1024 : 256);
+    cfg.blockDim = dim3(n > 256 ? 1024 : 256);      // one partial per thread up to 1024 CTAs: a single round trip
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
