@@ -298,7 +298,10 @@ db_status db_aggregate_update_host(db_host_pipeline* pipeline,
  *         bytes, 16-byte aligned, uninitialised.  Its first 32-bit word is a
  *         status word the call clears and the tensor-core kernels set to a
  *         non-zero code if one of their (time-limited) internal waits ever
- *         gives up; it stays 0 in correct operation.
+ *         gives up; it stays 0 in correct operation.  Calls enqueued on one
+ *         stream may share a workspace (none of a call's kernels touches it
+ *         before the previous call's have finished); calls that may overlap
+ *         on the device need distinct workspaces.
  *   flags 0, or DB_WORKER_GRAD_FFMA to run both contractions as plain fp32
  *         FFMA instead of on the tensor cores (the accuracy reference; also
  *         taken automatically for b_i > 4096)
