@@ -151,6 +151,36 @@ def test_equal_batches_are_the_plain_mean_and_k1_is_identity():
     assert torch.equal(v, g[0])
 
 
+@pytest.mark.parametrize("K", [2, 4, 8, 16])
+def test_equal_batches_with_k_a_power_of_two_are_the_fp32_mean_bit_for_bit(K):
+    """lambda = 1/K is then exact in fp32 and lambda * g_k exact too, so the kernel's chain
+    acc = fma(lambda, g_k, acc), k ascending from zero, is the left-to-right fp32 sum of the scaled gradients."""
+    N = 70_001
+    g = inputs.worker_gradients(K, N, 1.0, 81 + K, device=DEV)
+    p, v = torch.zeros(N, device=DEV), torch.zeros(N, device=DEV)
+    binding.aggregate_update(g, [24] * K, p, v, 1.0, 0.0)
+    acc = torch.zeros(N, device=DEV)
+    for gk in g:
+        acc = acc + gk * (1.0 / K)
+    assert torch.equal(v, acc) and torch.equal(p, -acc)
+
+
+def test_scaling_every_batch_size_changes_at_most_the_last_bit():
+    """b -> c b leaves the weights b_k / sum b unchanged as real numbers; formed in fp64 and rounded to fp32
+    they can differ in the last place at most, and so can the aggregate."""
+    N, K = 50_003, 5
+    g = inputs.worker_gradients(K, N, 1.0, 87, device=DEV)
+    b = [7, 13, 32, 58, 6]
+    outs = []
+    for c in (1, 3, 1000):
+        p, v = torch.zeros(N, device=DEV), torch.zeros(N, device=DEV)
+        binding.aggregate_update(g, [c * x for x in b], p, v, 1.0, 0.0)
+        outs.append(v)
+    scale = torch.stack([x.abs() for x in g]).amax(0)          # an ulp of the largest term bounds the change
+    for o in outs[1:]:
+        assert bool(((o - outs[0]).abs() <= K * scale * 2.0 ** -23).all())
+
+
 def test_norm_of_ones_is_exactly_N():
     N = 1_000_003
     ones = [torch.ones(N, device=DEV) for _ in range(4)]
