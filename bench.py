@@ -168,7 +168,7 @@ class ClockSampler:
     REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
                0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
 
-    def __init__(self, index: int, period_s: float = 0.001):
+    def __init__(self, index: int, period_s: float = 0.005):
         self.samples, self.reasons = [], set()
         self.max_mhz = None
         self._stop = threading.Event()
@@ -198,6 +198,10 @@ class ClockSampler:
     def _loop(self):
         nv = self.nv
         self._go.wait()
+        # An NVML query pair costs the running stream about 10 us (measured: a 20-step region of 3.5 ms sampled
+        # every millisecond ran 1 - 2.5 us per step slower than unsampled).  So: the first sample one millisecond
+        # into the region, then one every `period`.
+        self._stop.wait(0.001)
         while not self._stop.is_set():
             try:
                 self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
@@ -291,6 +295,9 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
         else:
             binding.aggregate_update(grads, b, p, v, wl.lr, wl.mu, sq, ws, stream)
 
+    # the sampler (NVML handle, thread) is set up before the warm-up steps, so that nothing but the barrier
+    # lies between the last warm-up step and the first timed one
+    sampler = ClockSampler(dev.index)
     warmup = max(3, args.warmup)
     for _ in range(warmup):
         step()
@@ -298,7 +305,6 @@ def measure(wl, args, dev, rank, world, with_e2e=True, with_cpu=True):
 
     # ---- timed region: device-resident inputs, one event before and one after all steps
     steps = args.steps
-    sampler = ClockSampler(dev.index)
     replicas.barrier(dev)
     torch.cuda.synchronize()
     if flush is None:
