@@ -3,8 +3,9 @@
 Each case below plants ONE plausible error in a copy of oracle/ref_oracle.c -- a dropped term, a wrong sign,
 a transposed operand, a missing normalisation -- builds the copy with the oracle's own compiler flags, and runs
 tests/test_oracle_pins.py against it in a child process (tests/oracle_mutation_runner.py; the oracle front end
-loads the library named by REF_ORACLE_LIB instead of building its own).  The pins must FAIL for every planted error and pass for an
-unaltered copy.  The errors live in the CPU oracle only; nothing here touches the CUDA library.
+loads the library named by REF_ORACLE_LIB instead of building its own).  The pins must FAIL for every planted
+error and pass for an unaltered copy.  The errors live in the CPU oracle only; nothing here touches the CUDA
+library.
 """
 import json
 import os
